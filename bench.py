@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the solve + verify path (gr_solve followed by gr_verify).
+
+One step = one pass of the whole path over one batch of synthetic instances of the
+headline workload (V=128256, n=8, draft top-k=50, batch 1024 per GPU, fp32 logits).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 it is launched by torch.distributed.run, one rank per GPU; every rank
+processes its own batch (instances are independent: no collective on the data path),
+the timed region is bracketed by barriers and the slowest rank's time is used.
+
+Prints one JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "solve+verify instances/sec at V=128256,n=8,top-k=50"
+UNIT = "instances/s"
+HEADLINE = dict(V=128256, n=8, topk=50, batch=1024, temp_target=0.7, temp_draft=1.0)
+BYTES_PER_INSTANCE = HEADLINE["V"] * (4 + 4)       # both fp32 logit rows, read once
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            parts = [x.strip() for x in r.split(",")]
+            if len(parts) < 6:
+                continue
+            try:
+                sm.append(float(parts[0])); smax = float(parts[1])
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[2:6]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        med = sm[len(sm) // 2] if sm else None
+        return {"sm_mhz": med, "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step solves + verifies a bounded sample."""
+    import numpy as np
+    import torch
+    from oracle import gr_oracle as O
+    from paper_2511_15898_b200 import workloads as W
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = 16
+    wl = W.config3(batch=sample, device="cpu", seed=3000)
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    tk = wl.draft_tokens.numpy(); un = wl.uniforms.numpy()
+    for _ in range(max(args.warmup, 0)):
+        O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, tk, un)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, tk, un)
+    dt = time.perf_counter() - t0
+    val = sample * args.steps / dt
+    cores = O.num_threads()
+    out = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config3: V=128256 n=8 top-k=50 fp32 logits, target temp 0.7, draft temp 1.0",
+                   "sample": f"{sample} instances per step (of the 1024-instance batch)"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": f"{sample} instances x {args.steps} steps, OpenMP over instances"},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out), flush=True)
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import paper_2511_15898_b200 as G
+    from paper_2511_15898_b200 import workloads as W
+    from paper_2511_15898_b200.build import build_library
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        build_library()
+    if world > 1:
+        dist.barrier()
+    G.load_library()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    H = HEADLINE
+    B = H["batch"]
+    wl = W.config3(batch=B, device=dev, seed=3000 + rank, V=H["V"], n=H["n"], topk=H["topk"])
+    ev_scan = torch.cuda.Event(enable_timing=True)
+    opt = G.Options(scan_done_event=ev_scan.cuda_event if hasattr(ev_scan, "cuda_event") else None)
+    solved = None
+    ver = None
+
+    def step(record=None):
+        nonlocal solved, ver
+        if record is not None:
+            record[0].record()
+        solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft, opt, solved)
+        if record is not None:
+            record[1].record()
+        ver = G.verify(solved, wl.draft_tokens, wl.uniforms, ver)
+        if record is not None:
+            record[2].record()
+
+    # torch creates the CUDA event lazily; recording it once makes its handle valid for the library
+    ev_scan.record()
+    opt.scan_done_event = ev_scan.cuda_event
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
+    scan_ms = []
+    start = torch.cuda.Event(enable_timing=True); end = torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(K):
+        step(evs[i])
+        # the scan-done event is re-recorded every step: read it before the next step overwrites it
+        evs[i][1].synchronize()
+        scan_ms.append(evs[i][0].elapsed_time(ev_scan))
+    end.record()
+    barrier()
+    total_ms = start.elapsed_time(end)
+    clocks = sampler.stop() if rank == 0 else None
+    solve_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    verify_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    step_ms = [e[0].elapsed_time(e[2]) for e in evs]
+    # the per-step sync above adds host gaps between steps; the step time is the device time of the two calls
+    dev_ms = float(np.sum(step_ms))
+    t = torch.tensor([dev_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dev_ms = float(t.item())
+    value = world * B * K / (dev_ms * 1e-3)
+
+    # ---- end to end through the public API with host (pinned) buffers
+    e2e = None
+    if rank == 0 or world > 1:
+        hq = wl.q_logits.cpu().pin_memory(); hp = wl.p_logits.cpu().pin_memory()
+        ht = wl.draft_tokens.cpu().pin_memory(); hu = wl.uniforms.cpu().pin_memory()
+        state = {}
+        Ke = max(2, min(K, 5))
+        for _ in range(2):
+            G.solve_verify_host(hq, hp, ht, hu, wl.n, wl.topk, wl.temp_target, wl.temp_draft, None, dev, state)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(Ke):
+            tok, acc, al, st = G.solve_verify_host(hq, hp, ht, hu, wl.n, wl.topk, wl.temp_target, wl.temp_draft,
+                                                   None, dev, state)
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        te = torch.tensor([dt], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        h2d = hq.numel() * hq.element_size() * 2 + ht.numel() * 4 + hu.numel() * 4
+        d2h = B * (4 + 1 + 4 + 4)
+        e2e = {"value": world * B * Ke / float(te.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "steps": Ke}
+        del hq, hp
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    scan_avg_ms = float(np.mean(scan_ms))
+    solve_avg_ms = float(np.mean(solve_ms))
+    ach = BYTES_PER_INSTANCE * B / (scan_avg_ms * 1e-3) / 1e9
+    path_gbs = BYTES_PER_INSTANCE * B / (float(np.mean(step_ms)) * 1e-3) / 1e9
+    status = solved.status.cpu().numpy()
+    acc_rate = float(ver.accepted.float().mean().item())
+
+    # ---- batch-1 call latency
+    wl1 = wl.rows([0])
+    s1 = None; v1 = None
+    lat = []
+    for i in range(30):
+        a = torch.cuda.Event(enable_timing=True); b_ = torch.cuda.Event(enable_timing=True)
+        a.record()
+        s1 = G.solve(wl1.q_logits, wl1.p_logits, wl1.n, wl1.topk, wl1.temp_target, wl1.temp_draft, None, s1)
+        v1 = G.verify(s1, wl1.draft_tokens, wl1.uniforms, v1)
+        b_.record(); b_.synchronize()
+        if i >= 10:
+            lat.append(a.elapsed_time(b_) * 1e3)
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload
+    from oracle import gr_oracle as O
+    ns = 32
+    sub = wl.rows(list(range(ns)))
+    tl = W.logits_to_f64(sub.q_logits); dl = W.logits_to_f64(sub.p_logits)
+    t0 = time.perf_counter()
+    O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, sub.draft_tokens.cpu().numpy(),
+                         sub.uniforms.cpu().numpy())
+    cpu_dt = time.perf_counter() - t0
+    cpu = {"value": ns / cpu_dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+           "sample": f"first {ns} instances of the batch, OpenMP over instances, {cpu_dt:.1f} s"}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "config3: V=128256 n=8 top-k=50 batch 1024 per GPU, fp32 logits, target temp 0.7, "
+                               "draft temp 1.0, Zipf-shaped logits", "global_batch": world * B,
+                   "cache": "inputs (1.05 GB per batch) larger than L2, no flush needed", "parallelism": f"batch x{world}"},
+        "roofline": {"bound": "hbm", "kernel": "scan_kernel (streams both logit rows once)", "achieved": ach,
+                     "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": None, "peak_kind": peak_kind,
+                     "kernel_ms": scan_avg_ms, "path_achieved": path_gbs, "path_frac": path_gbs / peak},
+        "kernels_ms": {"scan": scan_avg_ms, "solve": solve_avg_ms - scan_avg_ms, "verify": float(np.mean(verify_ms))},
+        "p50_us": {"batch_step": float(np.median(step_ms)) * 1e3,
+                   "per_instance_amortised": float(np.median(step_ms)) * 1e3 / B,
+                   "batch1_call": float(np.median(lat))},
+        "cpu_baseline": cpu,
+        "e2e": e2e,
+        "gpu_launches": 3 * K,
+        "clocks": clocks,
+        "quality": {"accept_rate": acc_rate, "status_ok": int((status == 0).sum()),
+                    "status_not_converged": int((status == 1).sum()), "wall_ms_total": total_ms},
+    }
+    print(json.dumps(out), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 8:
+            args.steps = 8       # bounded: a step is ~1 s of host time per 16 instances
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,169 @@
+/*
+ * gr.h -- C interface of the B200 (sm_100a) global-resolution library.
+ *
+ * For a batch of decode positions the library turns target logits, draft logits
+ * and the number n of i.i.d. drafts into the optimal-transport verification rule
+ * of "Global Resolution" (optimal multi-draft speculative sampling) and then
+ * draws the emitted token for the n drafted tokens.
+ *
+ * Letters.  The paper writes p for the target distribution and q for the draft
+ * distribution; this interface uses the opposite letters, as serving stacks do:
+ *   q_logits = TARGET model logits,  p_logits = DRAFT model logits.
+ * In the comments below "tgt" is the target distribution after temperature and
+ * "drf" the single-token draft distribution after temperature, top-k truncation
+ * and renormalisation (App. A, first paragraph; App. N).
+ *
+ * Conventions shared by every call
+ *   - every pointer named below is a DEVICE pointer owned by the caller unless
+ *     it is marked "host"; the library never allocates or frees device memory;
+ *   - calls only enqueue work on `stream` (a cudaStream_t passed as void*) and
+ *     return without synchronising;
+ *   - the int return value is 0 (GR_OK) when the work was enqueued, or a negative
+ *     GR_E_* code when the arguments were rejected on the host (nothing enqueued);
+ *   - data-dependent outcomes are reported per instance in the status arrays.
+ */
+#ifndef GR_H_
+#define GR_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* element type of the logits */
+#define GR_F32  0
+#define GR_BF16 1
+
+/* per-instance status values (status arrays, device memory) */
+#define GR_OK                    0
+#define GR_NOT_CONVERGED         1  /* iteration cap reached; the rule is usable, its gradient norm is in params */
+#define GR_SUPPORT_TOO_LARGE     2  /* support larger than GR_MAX_SUPPORT: no rule was solved; gr_verify falls
+                                       back to sampling the target distribution (still lossless), the paper's
+                                       "early termination" convention (Sec. 6.2 last paragraph, App. K)   */
+#define GR_BAD_LOGITS            3  /* a NaN or infinite logit in the row                                 */
+#define GR_DRAFT_OUT_OF_SUPPORT  4  /* a drafted token does not belong to the draft support               */
+#define GR_STALE_PARAMS          5  /* params block was not written by gr_solve for this shape            */
+
+/* host-side argument errors (return values) */
+#define GR_E_INVALID   (-1)  /* a size, temperature or option is out of range */
+#define GR_E_NULL      (-2)  /* a required pointer is NULL                    */
+#define GR_E_ALIGN     (-3)  /* a logits base pointer is not 16-byte aligned  */
+#define GR_E_LAUNCH    (-4)  /* the CUDA runtime refused a launch             */
+#define GR_E_TOO_LARGE (-5)  /* beyond a stated capacity                      */
+
+/* capacities */
+#define GR_MAX_SUPPORT 128   /* largest draft support for which the convex programs are solved */
+#define GR_MAX_DRAFTS  32    /* largest n                                                     */
+
+/*
+ * Solver options (host struct, read during the call).  NULL selects the defaults.
+ *   tol        stop when the L1 norm of the gradient of the convex function
+ *              (Theta for the inner system, Phi restricted to a block for the outer
+ *              system; Sec. 6.2) is <= tol.                      default 1e-9
+ *   max_iters  cap on gradient evaluations per system.            default 40
+ *   quad_step  step of the trapezoid rule in the log-time variable used to
+ *              evaluate the gradient integral; smaller is more accurate and
+ *              slower (error roughly exp(-pi^2/quad_step)).        default 0.4
+ *   scan_done_event  optional cudaEvent_t (as void*) recorded on `stream` between
+ *              the streaming kernel and the solve kernel, so that a caller can
+ *              time the two separately; NULL records nothing.      default NULL
+ */
+typedef struct gr_options {
+    double tol;
+    int    max_iters;
+    double quad_step;
+    void*  scan_done_event;
+} gr_options;
+
+/*
+ * Bytes of the opaque per-batch `params` block that gr_solve writes and
+ * gr_verify reads, and of the scratch `workspace` gr_solve needs while it runs.
+ * Both depend only on the shape.  Return 0 when the shape is invalid.
+ */
+size_t gr_params_bytes(int V, int n, int topk, int batch);
+size_t gr_workspace_bytes(int V, int n, int topk, int batch);
+
+/*
+ * gr_solve -- steps 1-3 of Algorithm 1 for every instance of the batch.
+ *
+ * Per instance (one decode position):
+ *   tgt = softmax(q_logits / temp_target) over the whole vocabulary;
+ *   support = the `topk` largest draft logits (equal logits: the smaller id is
+ *   kept), drf = softmax(p_logits / temp_draft) over the support (App. N);
+ *   H* and the optimal acceptance alpha* = 1 + min_H psi(H) by ordering the
+ *   support by decreasing drf/tgt and scanning prefixes (Eq. "subset-select",
+ *   Sec. 5.1; ties: smaller id first, shortest minimising prefix);
+ *   outer residuals by cumulative minima of psi along the increasing-ratio
+ *   chain (Sec. 6.1, Thm "polymatroid", Lemma "q-convex");
+ *   softmax parameters exp(alpha_i) of the inner system on H* (Thm "Inner
+ *   Convex Solver") and of every block of the outer system (Thm "Outer Convex
+ *   Solver" restricted to the tokens between two consecutive tight prefixes),
+ *   with the full truncation set T (tunable errors epsilon_T = gamma_T = 0).
+ *
+ * Arguments
+ *   q_logits, p_logits  [batch, V] row-major, dtype GR_F32 (float) or GR_BF16;
+ *                       base pointers 16-byte aligned; read only.
+ *   V >= 1, 1 <= n <= GR_MAX_DRAFTS, batch >= 0.
+ *   topk                1..V-1 truncates the draft; 0 or >= V keeps every id.
+ *   temp_target, temp_draft   > 0.
+ *   opt                 host pointer or NULL.
+ *   params              out, gr_params_bytes() bytes, 16-byte aligned.  It records
+ *                       the address of q_logits: gr_verify re-reads at most one
+ *                       1024-element chunk of a target row on the resample branch,
+ *                       so q_logits must stay unchanged until gr_verify has run.
+ *   workspace           scratch, gr_workspace_bytes() bytes, 16-byte aligned;
+ *                       contents are meaningless after the call completes.
+ *   alpha_star          out [batch] float, optimal acceptance probability.
+ *   status              out [batch] int, GR_OK / GR_NOT_CONVERGED /
+ *                       GR_SUPPORT_TOO_LARGE / GR_BAD_LOGITS.
+ */
+int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk,
+             float temp_target, float temp_draft, int batch, const gr_options* opt,
+             void* params, void* workspace, float* alpha_star, int* status, void* stream);
+
+/*
+ * gr_verify -- step 4 of Algorithm 1 (the slice pi(.|omega), Eqs. "cases" and
+ * "approx-c", normalised) and the draw of App. A steps 3-4.
+ *
+ * Per instance, U = distinct drafted tokens in order of first occurrence.
+ * If U lies in H*: pi(i) = w_i / (1 + sum_U w) and the rest, 1 / (1 + sum_U w), goes
+ * to the resample distribution (residuals / (1 - alpha*)); otherwise only the
+ * tokens of the lowest-ratio block met by U share the mass, pi(i) = w_i / sum w.
+ * The emitted token is the first segment (U's tokens in order, then the resample
+ * segment) whose cumulative probability exceeds u0; inside the resample segment
+ * it is the first id (ascending) whose cumulative residual exceeds u1 times the
+ * total residual.
+ *
+ *   params        written by gr_solve for the same batch; read only.
+ *   draft_tokens  [batch, n] int32 (n as given to gr_solve).
+ *   uniforms      [batch, 2] float in [0,1): (u0, u1).
+ *   out_token     out [batch] int32 emitted id, -1 on a per-instance error.
+ *   out_accepted  out [batch] 1 iff the emitted token is one of the drafts.
+ *   status        out [batch] GR_OK / GR_DRAFT_OUT_OF_SUPPORT / GR_STALE_PARAMS /
+ *                 GR_BAD_LOGITS, or the solve status when it was not GR_OK.
+ */
+int gr_verify(const void* params, const int* draft_tokens, const float* uniforms, int batch,
+              int* out_token, unsigned char* out_accepted, int* status, void* stream);
+
+/*
+ * gr_read_rule -- copies the rule of every instance out of `params` into plain
+ * arrays (for inspection and tests); all outputs are optional (NULL skips).
+ * Per-support arrays have `kcap` entries per instance and are filled in ratio
+ * order (position 0 = largest drf/tgt); unused entries are set to -1 / 0.
+ *   ids    [batch,kcap] int   token id          w   [batch,kcap] double exp(alpha_i)
+ *   block  [batch,kcap] int   -1 on H*, else block number counted from the lowest ratio
+ *   resid  [batch,kcap] double outer residual r_i (0 on H*)
+ *   flow   [batch,kcap] double p_i = tgt_i - r_i
+ *   header [batch,8] double: k, jstar, nblocks, alpha_star, gnorm, iterations, lse of the target row, status
+ */
+int gr_read_rule(const void* params, int batch, int kcap, int* ids, int* block, double* w,
+                 double* resid, double* flow, double* header, void* stream);
+
+/* Text for a GR_* / GR_E_* code (host pointer to a static string). */
+const char* gr_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GR_H_ */

@@ -1,0 +1,117 @@
+// Host side of the C interface declared in gr.h: argument checks and kernel launches.
+#include <math.h>
+#include "gr_common.cuh"
+
+namespace gr {
+void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
+                 double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
+int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
+                 cudaStream_t st);
+void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
+                   unsigned char* out_acc, int* status, cudaStream_t st);
+void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
+                      double* flow, double* header, cudaStream_t st);
+
+static bool shape_ok(int V, int n, int batch) {
+    return V >= 1 && V <= (1 << 21) && n >= 1 && n <= kMaxDrafts && batch >= 0;
+}
+}  // namespace gr
+
+extern "C" {
+
+size_t gr_params_bytes(int V, int n, int topk, int batch)
+{
+    if (!gr::shape_ok(V, n, batch)) return 0;
+    size_t s = (size_t)gr::params_stride(V, topk) * (size_t)(batch > 0 ? batch : 1);
+    return s;
+}
+
+size_t gr_workspace_bytes(int V, int n, int topk, int batch)
+{
+    if (!gr::shape_ok(V, n, batch)) return 0;
+    (void)topk;
+    return (size_t)gr::ws_stride() * (size_t)(batch > 0 ? batch : 1);
+}
+
+int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
+             float temp_draft, int batch, const gr_options* opt, void* params, void* workspace, float* alpha_star,
+             int* status, void* stream)
+{
+    if (!gr::shape_ok(V, n, batch)) return GR_E_INVALID;
+    if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
+    if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
+        return GR_E_INVALID;
+    double tol = 1e-9, qstep = 0.4;
+    int max_iters = 40;
+    cudaEvent_t scan_done = nullptr;
+    if (opt) {
+        scan_done = (cudaEvent_t)opt->scan_done_event;
+        tol = opt->tol; max_iters = opt->max_iters; qstep = opt->quad_step;
+        if (!(tol > 0.0) || max_iters < 1 || !(qstep >= 0.05 && qstep <= 2.0)) return GR_E_INVALID;
+    }
+    if (batch == 0) return GR_OK;
+    if (!q_logits || !p_logits || !params || !workspace || !alpha_star || !status) return GR_E_NULL;
+    if (((uintptr_t)q_logits & 15) || ((uintptr_t)p_logits & 15) || ((uintptr_t)params & 15) ||
+        ((uintptr_t)workspace & 15))
+        return GR_E_ALIGN;
+    const int kfull = (topk <= 0 || topk >= V) ? V : topk;
+    const int kcap = gr::kcap_of(V, topk);
+    const bool full_large = kcap == 0;
+    if (full_large && kfull != V) return GR_E_TOO_LARGE;   // a truncated support beyond the capacity
+    const int pstride = gr::params_stride(V, topk);
+    cudaStream_t st = (cudaStream_t)stream;
+    gr::launch_scan(q_logits, p_logits, dtype, V, kfull, full_large, (double)temp_target, (double)temp_draft, batch,
+                    (char*)workspace, (char*)params, pstride, kcap, st);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    int rc = gr::launch_solve((const char*)workspace, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
+                              (double)temp_draft, tol, max_iters, qstep, batch, alpha_star, status, st);
+    if (rc != GR_OK) return rc;
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    return GR_OK;
+}
+
+int gr_verify(const void* params, const int* draft_tokens, const float* uniforms, int batch, int* out_token,
+              unsigned char* out_accepted, int* status, void* stream)
+{
+    if (batch < 0) return GR_E_INVALID;
+    if (batch == 0) return GR_OK;
+    if (!params || !draft_tokens || !uniforms || !out_token || !out_accepted || !status) return GR_E_NULL;
+    if ((uintptr_t)params & 15) return GR_E_ALIGN;
+    gr::launch_verify((const char*)params, draft_tokens, uniforms, batch, out_token, out_accepted, status,
+                      (cudaStream_t)stream);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    return GR_OK;
+}
+
+int gr_read_rule(const void* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
+                 double* flow, double* header, void* stream)
+{
+    if (batch < 0 || kcap < 0) return GR_E_INVALID;
+    if (batch == 0) return GR_OK;
+    if (!params) return GR_E_NULL;
+    gr::launch_read_rule((const char*)params, batch, kcap, ids, block, w, resid, flow, header, (cudaStream_t)stream);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    return GR_OK;
+}
+
+const char* gr_strerror(int code)
+{
+    switch (code) {
+        case GR_OK: return "ok";
+        case GR_NOT_CONVERGED: return "iteration cap reached before the gradient tolerance";
+        case GR_SUPPORT_TOO_LARGE: return "draft support larger than GR_MAX_SUPPORT: rule not solved";
+        case GR_BAD_LOGITS: return "NaN or infinite logit";
+        case GR_DRAFT_OUT_OF_SUPPORT: return "drafted token outside the draft support";
+        case GR_STALE_PARAMS: return "params block was not written by gr_solve";
+        case GR_E_INVALID: return "invalid size, temperature or option";
+        case GR_E_NULL: return "required pointer is NULL";
+        case GR_E_ALIGN: return "pointer is not 16-byte aligned";
+        case GR_E_LAUNCH: return "CUDA launch failed";
+        case GR_E_TOO_LARGE: return "shape beyond the library's capacity";
+        default: return "unknown code";
+    }
+}
+
+}  // extern "C"

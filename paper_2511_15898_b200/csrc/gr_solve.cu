@@ -1,0 +1,574 @@
+// Per-instance solve (one CTA per instance): subset selection, outer residuals,
+// blocks, and the convex minimisation of the inner system and of every outer block.
+//
+// Gradient of the convex functions (Thm "Inner Convex Solver", Thm "Outer Convex
+// Solver"): with w_i = exp(alpha_i) the i-th gradient entry is g_i(w) - rhs_i,
+//   g_i = sum_{A containing i} Pr[set(omega) = A] w_i / (slack + sum_{j in A} w_j).
+// The exponentially many terms are summed exactly through
+//   1 / W = int_0^inf exp(-t W) dt   and   1 / W^2 = int_0^inf t exp(-t W) dt,
+// and the exponential generating function of n i.i.d. draws:  with x_j = exp(-t w_j),
+//   M(t) = n! [lambda^n] e^{lambda h} prod_j (1 + x_j (e^{lambda d_j} - 1)),
+//   g_i = w_i int e^{-t slack} x_i dM/dx_i dt,
+//   dg_i/dalpha_l = delta_il g_i - w_i w_l int t e^{-t slack} x_i x_l d2M/dx_i dx_l dt  (x_i for i = l),
+//   dM/dx_i = n! [lambda^n] P h_i,   d2M/dx_i dx_l = n! [lambda^n] P h_i h_l,
+//   P = e^{lambda h} prod_j f_j,  f_j = 1 + x_j e_j,  e_j = e^{lambda d_j} - 1,  h_j = e_j / f_j,
+// all as power series in lambda truncated at degree n.  The t-integral is a
+// trapezoid rule in s, t = exp(s - exp(-(s - s0))), which resolves every token's
+// transition at t ~ 1/w_j on a logarithmic scale and closes the lower tail
+// doubly exponentially.  Newton's method on alpha uses the exact Hessian above.
+#include "gr_common.cuh"
+
+namespace gr {
+
+constexpr int kSolveThreads = 256;
+constexpr int kSolveWarps = kSolveThreads / 32;
+constexpr int kGroups = 8;          // token groups whose partial products are combined per node
+constexpr double kTEnd = 25.0;      // integrand below exp(-kTEnd) at the upper end
+constexpr double kDrop = 1.0;       // the lower-tail compression starts this far below the fastest transition
+constexpr double kTail = 3.0;       // and the grid extends this far below that
+constexpr int kMaxNodes = 512;
+constexpr double kAlphaClamp = 80.0;
+constexpr double kStepClamp = 3.0;
+
+struct SolveLayout {
+    int KP, n, Qt;
+    // offsets in doubles
+    int d, tg, p, r, key, w, psi, Dr, alpha, alpha_prev, delta, g, g2, col, E, J, tq, cq, X, H, A, P, PP, gq, g2q, scal;
+    int ints;      // offset in bytes of the int region
+    int total_bytes;
+    __host__ __device__ SolveLayout(int KP_, int n_, int Qt_) : KP(KP_), n(n_), Qt(Qt_) {
+        int o = 0;
+        d = o; o += KP; tg = o; o += KP; p = o; o += KP; r = o; o += KP; key = o; o += KP; w = o; o += KP;
+        psi = o; o += KP + 4; Dr = o; o += KP + 4;
+        alpha = o; o += KP; alpha_prev = o; o += KP; delta = o; o += KP; g = o; o += KP; g2 = o; o += KP;
+        col = o; o += KP;
+        E = o; o += KP * (n + 1);
+        J = o; o += KP * (KP + 1) / 2;
+        tq = o; o += Qt; cq = o; o += Qt;
+        X = o; o += Qt * KP;
+        H = o; o += Qt * (n + 1) * KP;
+        A = o; o += Qt * (n + 1) * KP;
+        P = o; o += Qt * (n + 1);
+        PP = o; o += Qt * kGroups * (n + 1);
+        gq = o; o += Qt * KP; g2q = o; o += Qt * KP;
+        scal = o; o += 32;
+        ints = o * 8;
+        total_bytes = ints + KP * 4 * 4 + 64;
+    }
+};
+
+__host__ int solve_pick_tile(int KP, int n, int max_bytes) {
+    int Qt = 32;
+    while (Qt > 1 && SolveLayout(KP, n, Qt).total_bytes > max_bytes) Qt >>= 1;
+    return Qt;
+}
+__host__ int solve_smem_bytes(int KP, int n, int Qt) { return SolveLayout(KP, n, Qt).total_bytes; }
+
+struct Sm {
+    double *d, *tg, *p, *r, *key, *w, *psi, *Dr, *alpha, *alpha_prev, *delta, *g, *g2, *col, *E, *J, *tq, *cq, *X, *H,
+        *A, *P, *PP, *gq, *g2q, *scal;
+    int *id, *blk, *order, *itmp;
+    int KP, n, Qt;
+};
+
+__device__ inline int tri(int i, int l) { return i * (i + 1) / 2 + l; }   // l <= i
+
+// scal[] slots
+enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SHI, S_S0, S_STEP, S_H };
+
+__device__ double block_reduce_max(double v, double* scratch) {
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double r = scratch[0];
+    for (int i = 1; i < kSolveWarps; i++) r = fmax(r, scratch[i]);
+    return r;
+}
+__device__ double block_reduce_sum(double v, double* scratch) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double r = 0.0;
+    for (int i = 0; i < kSolveWarps; i++) r += scratch[i];
+    return r;
+}
+
+// Evaluate g (and, if want_jac, the packed lower triangle of the Hessian) at sm.alpha[0..m).
+// d = draft masses of the system's tokens, hmass = draft mass of everything of higher ratio
+// (outer blocks), slack = 1 for the inner system.  Returns the number of quadrature nodes.
+__device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, int slack, bool want_jac, double qstep)
+{
+    const int tid = threadIdx.x;
+    const int n = sm.n, n1 = sm.n + 1, KP = sm.KP, Qt = sm.Qt;
+    double* red = sm.scal + 16;
+    // weights and their range
+    double wj = 0.0;
+    if (tid < m) { wj = exp(sm.alpha[tid]); sm.w[tid] = wj; sm.g[tid] = 0.0; sm.g2[tid] = 0.0; }
+    double wmax = block_reduce_max(tid < m ? wj : 0.0, red);
+    double wmin = -block_reduce_max(tid < m ? -wj : -1.0e300, red);
+    if (want_jac)
+        for (int e = tid; e < m * (m + 1) / 2; e += kSolveThreads) sm.J[e] = 0.0;
+    const double rate = slack ? 1.0 + wmin : wmin;
+    const double s_hi = log(kTEnd / rate);
+    const double s0 = -log((slack ? 1.0 : 0.0) + wmax) - kDrop;
+    int Q = (int)ceil((s_hi - (s0 - kTail)) / qstep) + 1;
+    if (Q > kMaxNodes) Q = kMaxNodes;
+    double nfact = 1.0;
+    for (int c = 2; c <= n; c++) nfact *= (double)c;
+    const int gsz = (m + kGroups - 1) / kGroups;
+
+    for (int q0 = 0; q0 < Q; q0 += Qt) {
+        const int qn = min(Qt, Q - q0);
+        __syncthreads();
+        if (tid < qn) {
+            double s = s_hi - qstep * (double)(q0 + tid);
+            double e = exp(-(s - s0));
+            double t = exp(s - e);
+            double wt = qstep * (1.0 + e) * t;
+            sm.tq[tid] = t;
+            sm.cq[tid] = wt * (slack ? exp(-t) : 1.0) * nfact;
+        }
+        __syncthreads();
+        // per (node, token): survival x and the series h = e / (1 + x e)
+        for (int task = tid; task < qn * m; task += kSolveThreads) {
+            const int q = task / m, j = task - q * m;
+            const double x = exp(-sm.tq[q] * sm.w[j]);
+            sm.X[q * KP + j] = x;
+            double* Hq = sm.H + (size_t)q * n1 * KP;
+            for (int c = 1; c <= n; c++) {
+                double acc = 0.0;
+                for (int a = 1; a < c; a++) acc += sm.E[a * KP + j] * Hq[(c - a) * KP + j];
+                Hq[c * KP + j] = sm.E[c * KP + j] - x * acc;
+            }
+        }
+        // partial products of the factors f_j over token groups
+        for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
+            const int q = task / kGroups, grp = task - q * kGroups;
+            double* PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+            if (grp == 0) {
+                double hp = 1.0, fc = 1.0;
+                for (int c = 0; c <= n; c++) { PPq[c] = hp / fc; hp *= hmass; fc *= (double)(c + 1); }
+            } else {
+                PPq[0] = 1.0;
+                for (int c = 1; c <= n; c++) PPq[c] = 0.0;
+            }
+        }
+        __syncthreads();
+        for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
+            const int q = task / kGroups, grp = task - q * kGroups;
+            double* PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+            const int j0 = grp * gsz, j1 = min(m, j0 + gsz);
+            for (int j = j0; j < j1; j++) {
+                const double x = sm.X[q * KP + j];
+                for (int c = n; c >= 1; c--) {
+                    double acc = 0.0;
+                    for (int a = 1; a <= c; a++) acc += sm.E[a * KP + j] * PPq[c - a];
+                    PPq[c] += x * acc;
+                }
+            }
+        }
+        __syncthreads();
+        for (int stride = 1; stride < kGroups; stride <<= 1) {
+            for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
+                const int q = task / kGroups, grp = task - q * kGroups;
+                if ((grp % (2 * stride)) == 0 && grp + stride < kGroups) {
+                    double* Aq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+                    const double* Bq = sm.PP + (size_t)(q * kGroups + grp + stride) * n1;
+                    for (int c = n; c >= 0; c--) {
+                        double acc = 0.0;
+                        for (int a = 0; a <= c; a++) acc += Aq[a] * Bq[c - a];
+                        Aq[c] = acc;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        // per (node, token): gradient integrand; series A = P h scaled for the Hessian
+        for (int task = tid; task < qn * m; task += kSolveThreads) {
+            const int q = task / m, j = task - q * m;
+            const double* Pq = sm.PP + (size_t)(q * kGroups) * n1;
+            double* Hq = sm.H + (size_t)q * n1 * KP;
+            double val = 0.0;
+            for (int c = 1; c <= n; c++) val += Pq[n - c] * Hq[c * KP + j];
+            const double u = sm.w[j] * sm.X[q * KP + j];
+            const double cg = sm.cq[q];
+            const double gi = cg * u * val;
+            sm.gq[q * KP + j] = gi;
+            sm.g2q[q * KP + j] = gi * sm.tq[q] * sm.w[j];
+            if (want_jac) {
+                double* Aq = sm.A + (size_t)q * n1 * KP;
+                const double sa = cg * sm.tq[q] * u;
+                for (int e = 1; e < n; e++) {
+                    double acc = 0.0;
+                    for (int c = 1; c <= e; c++) acc += Hq[c * KP + j] * Pq[e - c];
+                    Aq[e * KP + j] = sa * acc;
+                }
+                for (int c = 1; c < n; c++) Hq[c * KP + j] *= u;
+            }
+        }
+        __syncthreads();
+        if (tid < m) {
+            double a = 0.0, b2 = 0.0;
+            for (int q = 0; q < qn; q++) { a += sm.gq[q * KP + tid]; b2 += sm.g2q[q * KP + tid]; }
+            sm.g[tid] += a; sm.g2[tid] += b2;
+        }
+        if (want_jac && n > 1) {
+            const int warp = tid >> 5, lane = tid & 31;
+            for (int i = 1 + warp; i < m; i += kSolveWarps) {
+                for (int l = lane; l < i; l += 32) {
+                    double acc = 0.0;
+                    for (int q = 0; q < qn; q++) {
+                        const double* Aq = sm.A + (size_t)q * n1 * KP;
+                        const double* Hq = sm.H + (size_t)q * n1 * KP;
+                        for (int c = 1; c < n; c++) acc += Aq[(n - c) * KP + i] * Hq[c * KP + l];
+                    }
+                    sm.J[tri(i, l)] -= acc;
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (want_jac && tid < m) sm.J[tri(tid, tid)] = sm.g[tid] - sm.g2[tid];
+    __syncthreads();
+    return Q;
+}
+
+// In-place Cholesky of the packed lower triangle; S_FAIL is set when a pivot is not positive.
+__device__ void cholesky(const Sm& sm, int m)
+{
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int j = 0; j < m; j++) {
+        __syncthreads();
+        const double pj = sm.J[tri(j, j)];
+        if (!(pj > 0.0)) { if (tid == 0) sm.scal[S_FAIL] = 1.0; __syncthreads(); return; }
+        const double inv = 1.0 / sqrt(pj);
+        for (int i = j + 1 + tid; i < m; i += kSolveThreads) sm.col[i] = sm.J[tri(i, j)] * inv;
+        __syncthreads();
+        if (tid == 0) sm.J[tri(j, j)] = sqrt(pj);
+        for (int i = j + 1 + tid; i < m; i += kSolveThreads) sm.J[tri(i, j)] = sm.col[i];
+        for (int i = j + 1 + warp; i < m; i += kSolveWarps) {
+            const double ci = sm.col[i];
+            for (int l = j + 1 + lane; l <= i; l += 32) sm.J[tri(i, l)] -= ci * sm.col[l];
+        }
+    }
+    __syncthreads();
+}
+
+// delta <- solution of L L^T delta = delta (one warp; column-oriented substitutions)
+__device__ void chol_solve(const Sm& sm, int m)
+{
+    const int tid = threadIdx.x;
+    if (tid < 32) {
+        const int lane = tid;
+        for (int i = 0; i < m; i++) {
+            if (lane == 0) sm.delta[i] = sm.delta[i] / sm.J[tri(i, i)];
+            __syncwarp();
+            const double yi = sm.delta[i];
+            for (int l = i + 1 + lane; l < m; l += 32) sm.delta[l] -= sm.J[tri(l, i)] * yi;
+            __syncwarp();
+        }
+        for (int i = m - 1; i >= 0; i--) {
+            if (lane == 0) sm.delta[i] = sm.delta[i] / sm.J[tri(i, i)];
+            __syncwarp();
+            const double xi = sm.delta[i];
+            for (int l = lane; l < i; l += 32) sm.delta[l] -= sm.J[tri(i, l)] * xi;
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+}
+
+// Newton iteration for one system.  On return sm.w[0..m) holds exp(alpha).
+// Returns the status; *gnorm and *iters receive the final L1 gradient norm and the evaluations spent.
+__device__ int solve_system(const Sm& sm, int m, const double* d, const double* rhs, double hmass, int slack,
+                            double tol, int max_iters, double qstep, double* gnorm, int* iters)
+{
+    const int tid = threadIdx.x, n = sm.n, KP = sm.KP;
+    double* red = sm.scal + 16;
+    // E[c][j] = d_j^c / c!
+    if (tid < m) {
+        double pw = 1.0, fc = 1.0;
+        sm.E[tid] = 0.0;
+        for (int c = 1; c <= n; c++) { pw *= d[tid]; fc *= (double)c; sm.E[c * KP + tid] = pw / fc; }
+    }
+    // starting point: the single-token balance  w/(1+w) * Pr[i in set(omega)] = rhs
+    double a0 = 0.0;
+    const double D = block_reduce_sum(tid < m ? d[tid] : 0.0, red);   // draft mass of the system
+    if (tid < m) {
+        if (slack) {
+            // Pr[i drafted and every draft inside the system] = D^n - (D - d_i)^n
+            double cap = pow(D, (double)n) - pow(fmax(D - d[tid], 0.0), (double)n);
+            double den = fmax(cap - rhs[tid], 1e-3 * rhs[tid]);
+            a0 = log(rhs[tid] / den);
+        } else {
+            a0 = log(rhs[tid] / d[tid]);
+        }
+    }
+    if (!slack) {
+        double mean = block_reduce_sum(tid < m ? a0 : 0.0, red) / (double)m;
+        a0 -= mean;
+    }
+    if (tid < m) sm.alpha[tid] = fmin(fmax(a0, -kAlphaClamp), kAlphaClamp);
+    if (tid == 0) { sm.scal[S_RPREV] = 1.0e300; sm.scal[S_LAM] = 1.0; }
+    __syncthreads();
+
+    int status = GR_NOT_CONVERGED;
+    int it = 0;
+    double rn = 0.0;
+    for (; it < max_iters; it++) {
+        eval_system(sm, m, d, hmass, slack, true, qstep);
+        rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
+        if (rn <= tol) { status = GR_OK; it++; break; }
+        const double rprev = sm.scal[S_RPREV];
+        const double lam = sm.scal[S_LAM];
+        __syncthreads();
+        if (!(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
+            // the last step did not reduce the gradient norm: retry it at half length
+            if (tid < m) sm.alpha[tid] = sm.alpha_prev[tid] + 0.5 * lam * sm.delta[tid];
+            if (tid == 0) sm.scal[S_LAM] = 0.5 * lam;
+            __syncthreads();
+            continue;
+        }
+        if (tid < m) sm.alpha_prev[tid] = sm.alpha[tid];
+        if (tid == 0) { sm.scal[S_RPREV] = rn; sm.scal[S_LAM] = 1.0; sm.scal[S_FAIL] = 0.0; }
+        if (!slack) {
+            // the block function is constant along (1,...,1): pin that direction
+            const double add = 1.0 / (double)m;
+            for (int e = tid; e < m * (m + 1) / 2; e += kSolveThreads) sm.J[e] += add;
+        }
+        __syncthreads();
+        cholesky(sm, m);
+        const bool fail = sm.scal[S_FAIL] != 0.0;
+        __syncthreads();
+        if (!fail) {
+            if (tid < m) sm.delta[tid] = -(sm.g[tid] - rhs[tid]);
+            __syncthreads();
+            chol_solve(sm, m);
+        } else {
+            // proportional-fitting step  alpha += log(rhs / g)
+            if (tid < m) sm.delta[tid] = log(rhs[tid] / sm.g[tid]);
+            __syncthreads();
+        }
+        double dm = block_reduce_max(tid < m ? fabs(sm.delta[tid]) : 0.0, red);
+        if (!(dm < 1.0e300)) dm = 1.0e300;
+        // a full Newton step below 1e-11 in alpha: the weights cannot be improved at this quadrature accuracy
+        if (!fail && dm < 1.0e-11) { status = GR_OK; it++; break; }
+        const double sc = dm > kStepClamp ? kStepClamp / dm : 1.0;
+        if (tid < m) {
+            double dl = sm.delta[tid] * sc;
+            if (!(dl == dl)) dl = 0.0;
+            sm.delta[tid] = dl;
+        }
+        __syncthreads();
+        double mean = 0.0;
+        if (!slack) mean = block_reduce_sum(tid < m ? sm.delta[tid] : 0.0, red) / (double)m;
+        if (tid < m) {
+            sm.delta[tid] -= mean;
+            double a = sm.alpha[tid] + sm.delta[tid];
+            sm.alpha[tid] = fmin(fmax(a, -kAlphaClamp), kAlphaClamp);
+        }
+        __syncthreads();
+    }
+    *gnorm = rn;
+    *iters = it;
+    return status;
+}
+
+__global__ void __launch_bounds__(kSolveThreads)
+solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
+             double temp_t, double temp_d, double tol, int max_iters, double qstep, int Qt,
+             float* __restrict__ alpha_out, int* __restrict__ status_out)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x;
+    const long long b = blockIdx.x;
+    char* pb = params + (size_t)b * pstride;
+    ParamView pv = view_params(pb, kcap);
+    const WsHeader* wh = reinterpret_cast<const WsHeader*>(ws + (size_t)b * ws_stride());
+    const int* w_id = reinterpret_cast<const int*>((const char*)wh + sizeof(WsHeader));
+    const float* w_dl = reinterpret_cast<const float*>(w_id + kMaxSupport);
+    const float* w_tl = w_dl + kMaxSupport;
+
+    const int kfull = (topk <= 0 || topk >= V) ? V : topk;
+    const int k = wh->count;
+    const bool bad = wh->bad != 0;
+    if (kcap == 0 || bad || k <= 0) {
+        // no rule: whole-vocabulary support beyond the capacity, or unusable logits
+        if (tid == 0) {
+            Header* h = pv.h;
+            h->n = n; h->k = 0; h->jstar = 0; h->nblocks = 0;
+            h->status = bad ? GR_BAD_LOGITS : GR_SUPPORT_TOO_LARGE;
+            h->alpha_star = __longlong_as_double(0x7ff8000000000000ll);
+            h->resid_total = 1.0; h->gnorm = 0.0; h->iters = 0;
+            __threadfence();
+            h->magic = kMagic;
+            alpha_out[b] = __int_as_float(0x7fc00000);
+            status_out[b] = h->status;
+        }
+        return;
+    }
+
+    const int KP = kcap;
+    SolveLayout L(KP, n, Qt);
+    double* base = reinterpret_cast<double*>(smem_raw);
+    Sm sm;
+    sm.d = base + L.d; sm.tg = base + L.tg; sm.p = base + L.p; sm.r = base + L.r; sm.key = base + L.key;
+    sm.w = base + L.w; sm.psi = base + L.psi; sm.Dr = base + L.Dr; sm.alpha = base + L.alpha;
+    sm.alpha_prev = base + L.alpha_prev; sm.delta = base + L.delta; sm.g = base + L.g; sm.g2 = base + L.g2;
+    sm.col = base + L.col; sm.E = base + L.E; sm.J = base + L.J; sm.tq = base + L.tq; sm.cq = base + L.cq;
+    sm.X = base + L.X; sm.H = base + L.H; sm.A = base + L.A; sm.P = base + L.P; sm.PP = base + L.PP;
+    sm.gq = base + L.gq; sm.g2q = base + L.g2q; sm.scal = base + L.scal;
+    int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
+    sm.id = ib; sm.blk = ib + KP; sm.order = ib + 2 * KP; sm.itmp = ib + 3 * KP;
+    sm.KP = KP; sm.n = n; sm.Qt = Qt;
+    double* red = sm.scal + 16;
+
+    const double lse_t = wh->lse_t;
+    // ---- distributions on the support (App. A; App. N): fp64 from the fp32 / bf16 logits
+    double a_i = 0.0, b_i = 0.0;
+    int my_id = 0;
+    if (tid < k) {
+        my_id = w_id[tid];
+        a_i = (double)w_tl[tid] / temp_t;
+        b_i = (double)w_dl[tid] / temp_d;
+    }
+    const double bmax = block_reduce_max(tid < k ? b_i : -1.0e300, red);
+    const double bsum = block_reduce_sum(tid < k ? exp(b_i - bmax) : 0.0, red);
+    const double lse_d = bmax + log(bsum);
+    // ---- ratio order: decreasing log-ratio key, equal keys by smaller id (Sec. 5.1)
+    if (tid < k) { sm.key[tid] = b_i - a_i; sm.itmp[tid] = my_id; }
+    __syncthreads();
+    if (tid < k) {
+        const double ky = sm.key[tid];
+        int rank = 0;
+        for (int j = 0; j < k; j++) {
+            const double kj = sm.key[j];
+            rank += (kj > ky || (kj == ky && sm.itmp[j] < my_id)) ? 1 : 0;
+        }
+        sm.id[rank] = my_id;
+        sm.tg[rank] = exp(a_i - lse_t);
+        sm.d[rank] = exp(b_i - lse_d);
+    }
+    __syncthreads();
+    // ---- prefix sums in order, psi along the chain, H* and alpha* (Eq. "subset-select")
+    if (tid == 0) {
+        double Tg = 0.0, Dr = 0.0;
+        sm.psi[0] = 0.0; sm.Dr[0] = 0.0;
+        for (int j = 1; j <= k; j++) {
+            Tg += sm.tg[j - 1]; Dr += sm.d[j - 1];
+            if (j == k) { Dr = 1.0; if (kfull == V) Tg = 1.0; }   // both distributions are normalised
+            sm.psi[j] = Tg; sm.Dr[j] = Dr;
+        }
+    }
+    __syncthreads();
+    if (tid >= 1 && tid <= k) sm.psi[tid] = sm.psi[tid] - pow(sm.Dr[tid], (double)n);
+    __syncthreads();
+    if (tid == 0) {
+        int jstar = 0; double best = 0.0;
+        for (int j = 1; j <= k; j++) if (sm.psi[j] < best) { best = sm.psi[j]; jstar = j; }
+        // ---- outer residuals by cumulative minima along the increasing-ratio chain; blocks end at
+        //      every new strict minimum (Sec. 6.1, Thm "polymatroid", Lemma "q-convex")
+        for (int j = 0; j < jstar; j++) { sm.p[j] = sm.tg[j]; sm.r[j] = 0.0; sm.blk[j] = -1; }
+        double m_prev = sm.psi[k];
+        int blk = 0, open = 0;
+        for (int s = 1; s <= k - jstar; s++) {
+            const int pos = k - s;
+            const double c = sm.psi[k - s];
+            const bool record = c < m_prev;
+            const double mm = record ? c : m_prev;
+            sm.r[pos] = m_prev - mm;
+            sm.p[pos] = sm.tg[pos] - sm.r[pos];
+            sm.blk[pos] = blk; open = 1;
+            if (record) { blk++; open = 0; }
+            m_prev = mm;
+        }
+        sm.scal[0] = (double)jstar;
+        sm.scal[1] = (double)(blk + open);
+        sm.scal[2] = 1.0 + best;
+    }
+    __syncthreads();
+    const int jstar = (int)sm.scal[0];
+    const int nblocks = (int)sm.scal[1];
+    const double alpha_star = sm.scal[2];
+    __syncthreads();
+
+    // ---- convex minimisation: inner system on H*, then every outer block with two or more tokens
+    int status = GR_OK, iters_total = 0;
+    double gnorm_total = 0.0;
+    if (tid < k) pv.w[tid] = 1.0;
+    if (jstar > 0) {
+        double gn; int it;
+        int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+        if (st != GR_OK) status = GR_NOT_CONVERGED;
+        gnorm_total += gn; iters_total += it;
+        if (tid < jstar) pv.w[tid] = sm.w[tid];
+        __syncthreads();
+    }
+    {
+        int lo = jstar;
+        while (lo < k) {
+            int hi = lo;
+            const int bk = sm.blk[lo];
+            while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
+            const int m = hi - lo + 1;
+            if (m >= 2) {
+                double gn; int it;
+                int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it);
+                if (st != GR_OK) status = GR_NOT_CONVERGED;
+                gnorm_total += gn; iters_total += it;
+                if (tid < m) pv.w[lo + tid] = sm.w[tid];
+                __syncthreads();
+            }
+            lo = hi + 1;
+        }
+    }
+
+    // ---- params
+    if (tid < KP) {
+        const bool in = tid < k;
+        pv.id[tid] = in ? sm.id[tid] : -1;
+        pv.blk[tid] = in ? sm.blk[tid] : -2;
+        pv.r[tid] = in ? sm.r[tid] : 0.0;
+        pv.p[tid] = in ? sm.p[tid] : 0.0;
+        if (!in) pv.w[tid] = 0.0;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        Header* h = pv.h;
+        h->n = n; h->k = k; h->jstar = jstar; h->nblocks = nblocks; h->status = status;
+        h->alpha_star = alpha_star;
+        h->resid_total = 1.0 - alpha_star;
+        h->gnorm = gnorm_total; h->iters = iters_total;
+        __threadfence();
+        h->magic = kMagic;
+        alpha_out[b] = (float)alpha_star;
+        status_out[b] = status;
+    }
+}
+
+int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
+                 cudaStream_t st)
+{
+    int Qt = 1, smem = 0;
+    if (kcap > 0) {
+        // keep several CTAs resident per SM when the shape allows it
+        Qt = solve_pick_tile(kcap, n, 72 * 1024);
+        if (solve_smem_bytes(kcap, n, Qt) > 72 * 1024) Qt = solve_pick_tile(kcap, n, 200 * 1024);
+        smem = solve_smem_bytes(kcap, n, Qt);
+        if (smem > 220 * 1024) return GR_E_TOO_LARGE;
+    }
+    static int configured = 0;
+    if (configured < smem) {
+        if (cudaFuncSetAttribute(solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
+            return GR_E_LAUNCH;
+        configured = 220 * 1024;
+    }
+    solve_kernel<<<batch, kSolveThreads, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
+                                                     max_iters, qstep, Qt, alpha_out, status_out);
+    return GR_OK;
+}
+
+}  // namespace gr

@@ -1,0 +1,169 @@
+"""Parity of the CUDA path (through the C interface) with the fp64 CPU oracle.
+
+Tolerances (the benchmark's stated ones): optimal acceptance within 1e-6 absolute,
+verification distribution within 1e-5 total variation, emitted tokens identical for
+identical uniforms except draws within 1e-6 of a CDF boundary.  Instances whose discrete
+structure hinges on a psi gap below 1e-6 are counted and excluded (see tests/parity.py).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2511_15898_b200 as G
+from paper_2511_15898_b200 import workloads as W
+from paper_2511_15898_b200.build import build_library
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+ALPHA_TOL = 1e-6
+TV_TOL = 1e-5
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build_library()
+    G.load_library()
+
+
+def _check(rep: P.Report, max_near_tie_frac=0.25):
+    print(rep.summary())
+    assert rep.alpha_err <= ALPHA_TOL, rep.summary()
+    assert rep.n_struct_mismatch == 0, (rep.summary(), rep.details[:5])
+    assert rep.tv <= TV_TOL, rep.summary()
+    assert rep.token_mismatch_other == 0, (rep.summary(), rep.details[:5])
+    assert rep.n_not_converged == 0, rep.summary()
+    assert rep.n_near_tie <= max_near_tie_frac * rep.n_inst, rep.summary()
+
+
+def test_config1_tiny_full_support():
+    _check(P.compare(W.config1(device="cuda")))
+
+
+def test_config2_top8():
+    _check(P.compare(W.config2(batch=64, device="cuda")))
+
+
+def test_config3_headline_shape():
+    _check(P.compare(W.config3(batch=24, device="cuda")))
+
+
+@pytest.mark.parametrize("n,topk,sigma", [(2, 5, 0.25), (4, 20, 1.0), (8, 5, 2.0), (16, 20, 0.25), (32, 5, 1.0),
+                                          (32, 20, 2.0)])
+def test_config4_topk_cells(n, topk, sigma):
+    _check(P.compare(W.config4(n, topk, sigma, batch=12, device="cuda")))
+
+
+def test_config5_bf16_top100():
+    _check(P.compare(W.config5(batch=4, device="cuda", rows_per_pass=4)))
+
+
+def test_ragged_rows_and_unaligned_vocabulary():
+    """V not a multiple of the vector width or of the chunk: scalar head / tail paths."""
+    for V, n, k in [(1031, 3, 6), (4099, 2, 4), (50257, 4, 5)]:
+        wl = W.config4(n, k, 1.0, batch=5, device="cuda", V=V, seed=77 + V)
+        _check(P.compare(wl))
+
+
+def test_full_batch_alpha_star_and_acceptance_properties():
+    """Headline size in the benchmark's launch configuration: properties that hold at any size,
+    and oracle values on sampled instances."""
+    wl = W.config3(batch=1024, device="cuda")
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+    ver = G.verify(solved, wl.draft_tokens, wl.uniforms)
+    torch.cuda.synchronize()
+    a = solved.alpha_star.cpu().numpy()
+    st = solved.status.cpu().numpy()
+    assert np.all(st == G.GR_OK)
+    assert np.all(a > 0) and np.all(a <= 1 + 1e-6)
+    tok = ver.token.cpu().numpy(); acc = ver.accepted.cpu().numpy()
+    dr = wl.draft_tokens.cpu().numpy()
+    in_draft = np.array([tok[b] in dr[b] for b in range(1024)])
+    assert np.array_equal(in_draft, acc.astype(bool))
+    assert np.all(tok >= 0) and np.all(tok < wl.V)
+    # acceptance frequency is near the mean optimal acceptance (binomial noise, 1024 draws)
+    assert abs(acc.mean() - a.mean()) < 5 * np.sqrt(0.25 / 1024)
+    idx = [0, 17, 333, 512, 1023]
+    rep = P.compare(wl.rows(idx))
+    _check(rep)
+    assert np.allclose(a[idx], solved.alpha_star[idx].cpu().numpy())
+
+
+def test_statuses_bad_logits_out_of_support_and_stale_params():
+    wl = W.config2(batch=4, device="cuda", V=5000)
+    q = wl.q_logits.clone(); p = wl.p_logits.clone()
+    q[1, 123] = float("nan")
+    p[2, 77] = float("inf")
+    solved = G.solve(q, p, wl.n, wl.topk)
+    toks = wl.draft_tokens.clone()
+    sup = torch.topk(wl.p_logits[3], 8).indices
+    outside = [i for i in range(100) if i not in sup.tolist()][0]
+    toks[3, 1] = outside
+    ver = G.verify(solved, toks, wl.uniforms)
+    torch.cuda.synchronize()
+    st = solved.status.cpu().tolist(); vs = ver.status.cpu().tolist(); tk = ver.token.cpu().tolist()
+    assert st[0] == G.GR_OK and st[1] == G.GR_BAD_LOGITS and st[2] == G.GR_BAD_LOGITS and st[3] == G.GR_OK
+    assert vs[0] == G.GR_OK and tk[0] >= 0
+    assert vs[1] == G.GR_BAD_LOGITS and tk[1] == -1
+    assert vs[3] == G.GR_DRAFT_OUT_OF_SUPPORT and tk[3] == -1
+    # a params block gr_solve never wrote
+    junk = G.binding.Solved(wl.V, wl.n, wl.topk, 4, torch.zeros_like(solved.params), solved.workspace,
+                            solved.alpha_star, solved.status, q)
+    ver2 = G.verify(junk, toks, wl.uniforms)
+    torch.cuda.synchronize()
+    assert ver2.status.cpu().tolist() == [G.GR_STALE_PARAMS] * 4 and ver2.token.cpu().tolist() == [-1] * 4
+
+
+def test_support_beyond_capacity_falls_back_to_target_sampling():
+    """Whole-vocabulary draft on a large vocabulary: no rule is solved (status says so) and
+    gr_verify emits a sample of the target distribution itself (inverse CDF at u1)."""
+    wl = W.config4(4, 0, 1.0, batch=6, device="cuda", V=5000, seed=99)
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk)
+    ver = G.verify(solved, wl.draft_tokens, wl.uniforms)
+    torch.cuda.synchronize()
+    assert solved.status.cpu().tolist() == [G.GR_SUPPORT_TOO_LARGE] * 6
+    tgt = torch.softmax(wl.q_logits.double(), dim=1).cpu().numpy()
+    u1 = wl.uniforms[:, 1].double().cpu().numpy()
+    tok = ver.token.cpu().numpy(); acc = ver.accepted.cpu().numpy()
+    for b in range(6):
+        cdf = np.cumsum(tgt[b])
+        want = int(np.searchsorted(cdf, u1[b] * cdf[-1], side="right"))
+        near = min(abs(cdf[want] - u1[b]), abs(cdf[max(want - 1, 0)] - u1[b])) < 1e-6
+        assert tok[b] == want or near
+        assert bool(acc[b]) == (tok[b] in wl.draft_tokens[b].cpu().tolist())
+
+
+def test_adversarial_row_order_takes_the_exact_selection_path():
+    """Strictly increasing draft logits defeat the streaming threshold (every element is a new
+    maximum); the candidate list overflows and the exact radix selection must give the same support."""
+    V, n, k, B = 40000, 3, 7, 3
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    q = torch.randn(B, V, generator=g, device="cuda")
+    p = torch.arange(V, device="cuda", dtype=torch.float32)[None, :].repeat(B, 1) * 1e-3
+    p[1] = p[1].flip(0)
+    p[2, ::2] = 0.5        # massive ties
+    wl0 = W.config2(batch=B, device="cuda", V=V)
+    toks = W.sample_draft_tokens(p, k, 1.0, n, g)
+    wl = W.Workload("adversarial", V, n, k, 1.0, 1.0, q.contiguous(), p.contiguous(), toks.contiguous(),
+                    wl0.uniforms)
+    _check(P.compare(wl), max_near_tie_frac=1.0)
+
+
+def test_repeat_calls_reuse_buffers_and_agree():
+    wl = W.config2(batch=16, device="cuda", V=9000)
+    s1 = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk)
+    v1 = G.verify(s1, wl.draft_tokens, wl.uniforms)
+    a1 = s1.alpha_star.clone(); t1 = v1.token.clone()
+    s2 = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, out=s1)
+    v2 = G.verify(s2, wl.draft_tokens, wl.uniforms, out=v1)
+    torch.cuda.synchronize()
+    assert torch.equal(a1, s2.alpha_star) and torch.equal(t1, v2.token)
+
+
+def test_host_buffer_front_end_matches_device_front_end():
+    wl = W.config2(batch=8, device="cuda", V=7000)
+    s = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk)
+    v = G.verify(s, wl.draft_tokens, wl.uniforms)
+    tok, acc, al, st = G.solve_verify_host(wl.q_logits.cpu(), wl.p_logits.cpu(), wl.draft_tokens.cpu(),
+                                           wl.uniforms.cpu(), wl.n, wl.topk)
+    assert torch.equal(tok, v.token.cpu()) and torch.equal(al, s.alpha_star.cpu())
