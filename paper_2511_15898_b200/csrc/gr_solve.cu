@@ -425,7 +425,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     sm.KP = KP; sm.n = n; sm.Qt = Qt;
     double* red = sm.scal + 16;
 
-    const double lse_t = wh->lse_t;
+    double lse_t = wh->lse_t;
     // ---- distributions on the support (App. A; App. N): fp64 from the fp32 / bf16 logits
     double a_i = 0.0, b_i = 0.0;
     int my_id = 0;
@@ -437,6 +437,15 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     const double bmax = block_reduce_max(tid < k ? b_i : -1.0e300, red);
     const double bsum = block_reduce_sum(tid < k ? exp(b_i - bmax) : 0.0, red);
     const double lse_d = bmax + log(bsum);
+    if (kfull == V) {
+        // the support is the whole vocabulary: normalise the target in fp64 over these same entries, so that
+        // it sums to one to rounding (the streaming kernel's fp32 sum is only good to ~1e-7, which would
+        // leave the outermost block's flows inconsistent with the mass of the tuples that feed them)
+        const double amax = block_reduce_max(tid < k ? a_i : -1.0e300, red);
+        const double asum = block_reduce_sum(tid < k ? exp(a_i - amax) : 0.0, red);
+        lse_t = amax + log(asum);
+        if (tid == 0) pv.h->lse_t = lse_t;
+    }
     // ---- ratio order: decreasing log-ratio key, equal keys by smaller id (Sec. 5.1)
     if (tid < k) { sm.key[tid] = b_i - a_i; sm.itmp[tid] = my_id; }
     __syncthreads();
