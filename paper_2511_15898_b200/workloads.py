@@ -32,6 +32,12 @@ class Workload:
     draft_tokens: torch.Tensor  # [B, n] int32, i.i.d. draws from the truncated draft distribution
     uniforms: torch.Tensor      # [B, 2] fp32 in [0, 1): verification uniforms (u0, u1)
 
+    def __post_init__(self):
+        # the C interface takes the temperatures as float: keep exactly those values, so that every
+        # consumer of the workload (CUDA path, CPU oracle) divides by the same numbers
+        self.temp_target = float(torch.tensor(self.temp_target, dtype=torch.float32).item())
+        self.temp_draft = float(torch.tensor(self.temp_draft, dtype=torch.float32).item())
+
     @property
     def batch(self) -> int:
         return self.q_logits.shape[0]
