@@ -123,6 +123,33 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
              void* params, void* workspace, float* alpha_star, int* status, void* stream);
 
 /*
+ * gr_solve_static -- gr_solve without the `workspace` argument, for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this is an interface variant.)
+ *
+ * Who needs it: a serving loop that has handed all free device memory to its own pool
+ * (KV cache, activation arena) and therefore must not call cudaMalloc at steady state --
+ * the call may fail there and it synchronises the whole device -- or a host that is not
+ * allowed to allocate at all once it is running (latency-bounded control loops).  Such a
+ * caller still owns `params` and the outputs, but has nowhere to take scratch from.
+ *
+ * The scratch is a fixed array inside the library's device image, GR_STATIC_MAX_BATCH
+ * instances large (about 0.4 MB, held by every GPU that loads the library until exit).
+ *   - batch > GR_STATIC_MAX_BATCH returns GR_E_TOO_LARGE and launches nothing; split the batch.
+ *   - The first call on each device looks the array's device address up (that device must
+ *     be current, as for any launch); make that first call before any stream capture.
+ *   - The call itself allocates and frees nothing.
+ *   - All calls share the one array and it keeps the previous call's contents.  Nothing in it
+ *     needs clearing (each call rewrites all it reads), but two calls whose kernels overlap on
+ *     the GPU -- different streams, or different host threads -- race on it: serialise them.
+ * Every other argument, the outputs and the statuses are exactly those of gr_solve, and
+ * gr_verify / gr_read_rule take the resulting `params` unchanged.
+ */
+#define GR_STATIC_MAX_BATCH 256
+int gr_solve_static(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk,
+                    float temp_target, float temp_draft, int batch, const gr_options* opt,
+                    void* params, float* alpha_star, int* status, void* stream);
+
+/*
  * gr_verify -- step 4 of Algorithm 1 (the slice pi(.|omega), Eqs. "cases" and
  * "approx-c", normalised) and the draw of App. A steps 3-4.
  *

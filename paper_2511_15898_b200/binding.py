@@ -18,6 +18,7 @@ import torch
 GR_F32, GR_BF16 = 0, 1
 GR_OK, GR_NOT_CONVERGED, GR_SUPPORT_TOO_LARGE, GR_BAD_LOGITS, GR_DRAFT_OUT_OF_SUPPORT, GR_STALE_PARAMS = range(6)
 GR_MAX_SUPPORT, GR_MAX_DRAFTS = 128, 32
+GR_STATIC_MAX_BATCH = 256
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgr_b200.so")
@@ -56,6 +57,9 @@ def load_library():
     lib.gr_solve.restype = C.c_int
     lib.gr_solve.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int,
                              C.POINTER(Options), vp, vp, fp, ip, vp]
+    lib.gr_solve_static.restype = C.c_int
+    lib.gr_solve_static.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int,
+                                    C.POINTER(Options), vp, fp, ip, vp]
     lib.gr_verify.restype = C.c_int
     lib.gr_verify.argtypes = [vp, ip, fp, C.c_int, ip, vp, ip, vp]
     lib.gr_read_rule.restype = C.c_int
@@ -86,6 +90,16 @@ def gr_solve(q_logits: int, p_logits: int, dtype: int, V: int, n: int, topk: int
     return int(load_library().gr_solve(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch,
                                        C.byref(opt) if opt is not None else None, params, workspace, alpha_star,
                                        status, stream))
+
+
+def gr_solve_static(q_logits: int, p_logits: int, dtype: int, V: int, n: int, topk: int, temp_target: float,
+                    temp_draft: float, batch: int, opt: Optional[Options], params: int, alpha_star: int, status: int,
+                    stream: int) -> int:
+    """gr_solve with the scratch inside the library (at most GR_STATIC_MAX_BATCH instances): for callers that
+    must not allocate device memory.  Calls that overlap on the GPU share that scratch and race."""
+    return int(load_library().gr_solve_static(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch,
+                                              C.byref(opt) if opt is not None else None, params, alpha_star, status,
+                                              stream))
 
 
 def gr_verify(params: int, draft_tokens: int, uniforms: int, batch: int, out_token: int, out_accepted: int,
