@@ -68,12 +68,16 @@ extern "C" {
  *   scan_done_event  optional cudaEvent_t (as void*) recorded on `stream` between
  *              the streaming kernel and the solve kernel, so that a caller can
  *              time the two separately; NULL records nothing.      default NULL
+ *   force_robust  non-zero sends every shape to the general (slower) solve kernel;
+ *              by default supports of at most 64 tokens with n <= 8 take a faster
+ *              kernel that computes the same rule.                  default 0
  */
 typedef struct gr_options {
     double tol;
     int    max_iters;
     double quad_step;
     void*  scan_done_event;
+    int    force_robust;
 } gr_options;
 
 /*

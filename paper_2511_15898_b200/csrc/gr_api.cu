@@ -6,12 +6,30 @@ namespace gr {
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                 cudaStream_t st);
+                 double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
+                 int* status_out, cudaStream_t st);
+int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
+                cudaStream_t st);
 void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
                    unsigned char* out_acc, int* status, cudaStream_t st);
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
                       double* flow, double* header, cudaStream_t st);
+
+// The fast kernel covers supports up to 64 tokens with n <= 8; everything else, and any instance the fast
+// kernel could not finish, takes the robust kernel.
+int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                     double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
+                     float* alpha_out, int* status_out, cudaStream_t st)
+{
+    int rc = force_robust ? 1
+                          : launch_fast(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep,
+                                        batch, alpha_out, status_out, st);
+    if (rc < 0) return rc;
+    // rc == 1: no fast variant, the robust kernel does everything; rc == 0: it redoes what the fast one flagged
+    return launch_solve(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch,
+                        rc == 0 ? 1 : 0, alpha_out, status_out, st);
+}
 
 static bool shape_ok(int V, int n, int batch) {
     return V >= 1 && V <= (1 << 21) && n >= 1 && n <= kMaxDrafts && batch >= 0;
@@ -45,8 +63,10 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
     double tol = 1e-9, qstep = 0.4;
     int max_iters = 40;
     cudaEvent_t scan_done = nullptr;
+    int force_robust = 0;
     if (opt) {
         scan_done = (cudaEvent_t)opt->scan_done_event;
+        force_robust = opt->force_robust;
         tol = opt->tol; max_iters = opt->max_iters; qstep = opt->quad_step;
         if (!(tol > 0.0) || max_iters < 1 || !(qstep >= 0.05 && qstep <= 2.0)) return GR_E_INVALID;
     }
@@ -65,8 +85,9 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
                     (char*)workspace, (char*)params, pstride, kcap, st);
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
-    int rc = gr::launch_solve((const char*)workspace, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
-                              (double)temp_draft, tol, max_iters, qstep, batch, alpha_star, status, st);
+    int rc = gr::launch_solve_any((const char*)workspace, (char*)params, pstride, kcap, V, n, topk,
+                                  (double)temp_target, (double)temp_draft, tol, max_iters, qstep, batch, force_robust,
+                                  alpha_star, status, st);
     if (rc != GR_OK) return rc;
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;

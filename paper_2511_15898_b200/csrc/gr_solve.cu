@@ -16,7 +16,7 @@
 // trapezoid rule in s, t = exp(s - exp(-(s - s0))), which resolves every token's
 // transition at t ~ 1/w_j on a logarithmic scale and closes the lower tail
 // doubly exponentially.  Newton's method on alpha uses the exact Hessian above.
-#include "gr_common.cuh"
+#include "gr_prep.cuh"
 
 namespace gr {
 
@@ -75,25 +75,6 @@ __device__ inline int tri(int i, int l) { return i * (i + 1) / 2 + l; }   // l <
 
 // scal[] slots
 enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SHI, S_S0, S_STEP, S_H };
-
-__device__ double block_reduce_max(double v, double* scratch) {
-    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double r = scratch[0];
-    for (int i = 1; i < kSolveWarps; i++) r = fmax(r, scratch[i]);
-    return r;
-}
-__device__ double block_reduce_sum(double v, double* scratch) {
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
-    __syncthreads();
-    double r = 0.0;
-    for (int i = 0; i < kSolveWarps; i++) r += scratch[i];
-    return r;
-}
 
 // Evaluate g (and, if want_jac, the packed lower triangle of the Hessian) at sm.alpha[0..m).
 // d = draft masses of the system's tokens, hmass = draft mass of everything of higher ratio
@@ -378,7 +359,7 @@ __device__ int solve_system(const Sm& sm, int m, const double* d, const double* 
 
 __global__ void __launch_bounds__(kSolveThreads)
 solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
-             double temp_t, double temp_d, double tol, int max_iters, double qstep, int Qt,
+             double temp_t, double temp_d, double tol, int max_iters, double qstep, int Qt, int only_flagged,
              float* __restrict__ alpha_out, int* __restrict__ status_out)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -386,27 +367,12 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     const long long b = blockIdx.x;
     char* pb = params + (size_t)b * pstride;
     ParamView pv = view_params(pb, kcap);
-    const WsHeader* wh = reinterpret_cast<const WsHeader*>(ws + (size_t)b * ws_stride());
-    const int* w_id = reinterpret_cast<const int*>((const char*)wh + sizeof(WsHeader));
-    const float* w_dl = reinterpret_cast<const float*>(w_id + kMaxSupport);
-    const float* w_tl = w_dl + kMaxSupport;
-
-    const int kfull = (topk <= 0 || topk >= V) ? V : topk;
-    const int k = wh->count;
-    const bool bad = wh->bad != 0;
-    if (kcap == 0 || bad || k <= 0) {
+    const WsView wv = view_ws(ws, b);
+    // second pass after the fast kernel: only the instances it flagged are redone
+    if (only_flagged && !(pv.h->magic == kMagic && pv.h->status == kNeedFallback)) return;
+    if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
         // no rule: whole-vocabulary support beyond the capacity, or unusable logits
-        if (tid == 0) {
-            Header* h = pv.h;
-            h->n = n; h->k = 0; h->jstar = 0; h->nblocks = 0;
-            h->status = bad ? GR_BAD_LOGITS : GR_SUPPORT_TOO_LARGE;
-            h->alpha_star = __longlong_as_double(0x7ff8000000000000ll);
-            h->resid_total = 1.0; h->gnorm = 0.0; h->iters = 0;
-            __threadfence();
-            h->magic = kMagic;
-            alpha_out[b] = __int_as_float(0x7fc00000);
-            status_out[b] = h->status;
-        }
+        if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
         return;
     }
 
@@ -425,83 +391,11 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     sm.KP = KP; sm.n = n; sm.Qt = Qt;
     double* red = sm.scal + 16;
 
-    double lse_t = wh->lse_t;
-    // ---- distributions on the support (App. A; App. N): fp64 from the fp32 / bf16 logits
-    double a_i = 0.0, b_i = 0.0;
-    int my_id = 0;
-    if (tid < k) {
-        my_id = w_id[tid];
-        a_i = (double)w_tl[tid] / temp_t;
-        b_i = (double)w_dl[tid] / temp_d;
-    }
-    const double bmax = block_reduce_max(tid < k ? b_i : -1.0e300, red);
-    const double bsum = block_reduce_sum(tid < k ? exp(b_i - bmax) : 0.0, red);
-    const double lse_d = bmax + log(bsum);
-    if (kfull == V) {
-        // the support is the whole vocabulary: normalise the target in fp64 over these same entries, so that
-        // it sums to one to rounding (the streaming kernel's fp32 sum is only good to ~1e-7, which would
-        // leave the outermost block's flows inconsistent with the mass of the tuples that feed them)
-        const double amax = block_reduce_max(tid < k ? a_i : -1.0e300, red);
-        const double asum = block_reduce_sum(tid < k ? exp(a_i - amax) : 0.0, red);
-        lse_t = amax + log(asum);
-        if (tid == 0) pv.h->lse_t = lse_t;
-    }
-    // ---- ratio order: decreasing log-ratio key, equal keys by smaller id (Sec. 5.1)
-    if (tid < k) { sm.key[tid] = b_i - a_i; sm.itmp[tid] = my_id; }
-    __syncthreads();
-    if (tid < k) {
-        const double ky = sm.key[tid];
-        int rank = 0;
-        for (int j = 0; j < k; j++) {
-            const double kj = sm.key[j];
-            rank += (kj > ky || (kj == ky && sm.itmp[j] < my_id)) ? 1 : 0;
-        }
-        sm.id[rank] = my_id;
-        sm.tg[rank] = exp(a_i - lse_t);
-        sm.d[rank] = exp(b_i - lse_d);
-    }
-    __syncthreads();
-    // ---- prefix sums in order, psi along the chain, H* and alpha* (Eq. "subset-select")
-    if (tid == 0) {
-        double Tg = 0.0, Dr = 0.0;
-        sm.psi[0] = 0.0; sm.Dr[0] = 0.0;
-        for (int j = 1; j <= k; j++) {
-            Tg += sm.tg[j - 1]; Dr += sm.d[j - 1];
-            if (j == k) { Dr = 1.0; if (kfull == V) Tg = 1.0; }   // both distributions are normalised
-            sm.psi[j] = Tg; sm.Dr[j] = Dr;
-        }
-    }
-    __syncthreads();
-    if (tid >= 1 && tid <= k) sm.psi[tid] = sm.psi[tid] - pow(sm.Dr[tid], (double)n);
-    __syncthreads();
-    if (tid == 0) {
-        int jstar = 0; double best = 0.0;
-        for (int j = 1; j <= k; j++) if (sm.psi[j] < best) { best = sm.psi[j]; jstar = j; }
-        // ---- outer residuals by cumulative minima along the increasing-ratio chain; blocks end at
-        //      every new strict minimum (Sec. 6.1, Thm "polymatroid", Lemma "q-convex")
-        for (int j = 0; j < jstar; j++) { sm.p[j] = sm.tg[j]; sm.r[j] = 0.0; sm.blk[j] = -1; }
-        double m_prev = sm.psi[k];
-        int blk = 0, open = 0;
-        for (int s = 1; s <= k - jstar; s++) {
-            const int pos = k - s;
-            const double c = sm.psi[k - s];
-            const bool record = c < m_prev;
-            const double mm = record ? c : m_prev;
-            sm.r[pos] = m_prev - mm;
-            sm.p[pos] = sm.tg[pos] - sm.r[pos];
-            sm.blk[pos] = blk; open = 1;
-            if (record) { blk++; open = 0; }
-            m_prev = mm;
-        }
-        sm.scal[0] = (double)jstar;
-        sm.scal[1] = (double)(blk + open);
-        sm.scal[2] = 1.0 + best;
-    }
-    __syncthreads();
-    const int jstar = (int)sm.scal[0];
-    const int nblocks = (int)sm.scal[1];
-    const double alpha_star = sm.scal[2];
-    __syncthreads();
+    PrepSm ps;
+    ps.d = sm.d; ps.tg = sm.tg; ps.p = sm.p; ps.r = sm.r; ps.key = sm.key; ps.psi = sm.psi; ps.Dr = sm.Dr;
+    ps.id = sm.id; ps.blk = sm.blk; ps.itmp = sm.itmp; ps.red = red; ps.out3 = sm.scal;
+    const PrepResult pr = prep_instance(ps, wv, pv.h, V, n, topk, temp_t, temp_d);
+    const int k = pr.k, jstar = pr.jstar;
 
     // ---- convex minimisation: inner system on H*, then every outer block with two or more tokens
     int status = GR_OK, iters_total = 0;
@@ -534,32 +428,12 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
         }
     }
 
-    // ---- params
-    if (tid < KP) {
-        const bool in = tid < k;
-        pv.id[tid] = in ? sm.id[tid] : -1;
-        pv.blk[tid] = in ? sm.blk[tid] : -2;
-        pv.r[tid] = in ? sm.r[tid] : 0.0;
-        pv.p[tid] = in ? sm.p[tid] : 0.0;
-        if (!in) pv.w[tid] = 0.0;
-    }
-    __syncthreads();
-    if (tid == 0) {
-        Header* h = pv.h;
-        h->n = n; h->k = k; h->jstar = jstar; h->nblocks = nblocks; h->status = status;
-        h->alpha_star = alpha_star;
-        h->resid_total = 1.0 - alpha_star;
-        h->gnorm = gnorm_total; h->iters = iters_total;
-        __threadfence();
-        h->magic = kMagic;
-        alpha_out[b] = (float)alpha_star;
-        status_out[b] = status;
-    }
+    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
 }
 
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                 cudaStream_t st)
+                 double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
+                 int* status_out, cudaStream_t st)
 {
     int Qt = 1, smem = 0;
     if (kcap > 0) {
@@ -576,7 +450,7 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
         configured = 220 * 1024;
     }
     solve_kernel<<<batch, kSolveThreads, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
-                                                     max_iters, qstep, Qt, alpha_out, status_out);
+                                                     max_iters, qstep, Qt, only_flagged, alpha_out, status_out);
     return GR_OK;
 }
 

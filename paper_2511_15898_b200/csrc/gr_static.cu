@@ -8,9 +8,9 @@
 namespace gr {
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
-int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                 cudaStream_t st);
+int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                     double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
+                     float* alpha_out, int* status_out, cudaStream_t st);
 
 constexpr int kStaticBytes = GR_STATIC_MAX_BATCH * (int)(sizeof(WsHeader) + kMaxSupport * 12);
 
@@ -51,8 +51,10 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     double tol = 1e-9, qstep = 0.4;
     int max_iters = 40;
     cudaEvent_t scan_done = nullptr;
+    int force_robust = 0;
     if (opt) {
         scan_done = (cudaEvent_t)opt->scan_done_event;
+        force_robust = opt->force_robust;
         tol = opt->tol; max_iters = opt->max_iters; qstep = opt->quad_step;
         if (!(tol > 0.0) || max_iters < 1 || !(qstep >= 0.05 && qstep <= 2.0)) return GR_E_INVALID;
     }
@@ -73,8 +75,9 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
                     ws, (char*)params, pstride, kcap, st);
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
-    const int rc = gr::launch_solve(ws, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
-                                    (double)temp_draft, tol, max_iters, qstep, batch, alpha_star, status, st);
+    const int rc = gr::launch_solve_any(ws, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
+                                        (double)temp_draft, tol, max_iters, qstep, batch, force_robust, alpha_star,
+                                        status, st);
     if (rc != GR_OK) return rc;
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;
