@@ -34,7 +34,6 @@ constexpr double kFTail = 3.0;
 constexpr int kFMaxNodes = 128;
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
-constexpr int kJLD = kMP + 1;         // leading dimension of the fp64 Hessian
 
 struct FastLayout {
     int KP;
@@ -50,9 +49,9 @@ struct FastLayout {
         tq = o; o += kFMaxNodes; cq = o; o += kFMaxNodes;
         scal = o; o += 32;
         uni = o;
-        // union: staging of the Hessian operands (two float arrays [kJC][NT-1][kMP]) / the fp64 Hessian
+        // union: staging of the Hessian operands (two float arrays [kJC][NT-1][kMP]) / elimination buffers
         const int stage_doubles = (2 * kJC * (NT - 1) * kMP * 4 + 7) / 8;
-        const int jmat_doubles = kMP * kJLD;
+        const int jmat_doubles = 2 * (kMP + 2) + 2 * kMP;    // pivot row / column buffers of the elimination
         o += stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
         jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
         o += kMP * kMP / 2;
@@ -338,48 +337,92 @@ __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
     __syncthreads();
 }
 
-// In-place Cholesky of the lower triangle of sm.J (leading dimension kJLD); thread i owns row i.
-// SC_FAIL is set when a pivot is not positive.
-__device__ void fast_cholesky(const FSm& sm, int m)
+// Newton step by Gauss-Jordan elimination without pivoting (the Hessian is symmetric positive
+// definite) on the matrix held in registers: thread (ty, tx) = (tid / 8, tid % 8) owns the entries
+// (i, l) with i = ty + 16 r, l = tx + 8 c, and the right-hand side of its rows when tx == 0.  Every
+// step publishes the pivot row and the pivot column through double-buffered shared memory, so it
+// costs one CTA barrier; after m steps the right-hand side holds the solution, with no triangular
+// substitutions.  Entries: off-diagonal -Jacc (lower triangle stored), diagonal g - g2, plus `add`
+// everywhere.  Writes the step into sm.delta; sets SC_FAIL when a pivot is not positive.
+__device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
 {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, ty = tid >> 3, tx = tid & 7;
+    double a[4][8], bb[4];
+    double* rowbuf = sm.J;                 // [2][kMP + 2]
+    double* colbuf = sm.J + 2 * (kMP + 2); // [2][kMP]
+#pragma unroll
+    for (int r = 0; r < 4; r++) {
+        const int i = ty + 16 * r;
+#pragma unroll
+        for (int c = 0; c < 8; c++) {
+            const int l = tx + 8 * c;
+            double v;
+            if (i < m && l < m) {
+                if (i == l) v = sm.g[i] - sm.g2[i];
+                else v = -(double)(i > l ? sm.Jacc[i * kMP + l] : sm.Jacc[l * kMP + i]);
+                v += add;
+            } else {
+                v = (i == l) ? 1.0 : 0.0;
+            }
+            a[r][c] = v;
+        }
+        bb[r] = i < m ? -(sm.g[i] - rhs[i]) : 0.0;
+    }
+    __syncthreads();     // everyone has read Jacc / g before the buffers (which alias the staging area) are written
+    bool bad = false;
     for (int j = 0; j < m; j++) {
+        const int pp = j & 1;
+        double* rb = rowbuf + pp * (kMP + 2);
+        double* cb = colbuf + pp * kMP;
+        const int rj = j >> 4, cj = j >> 3;
+        if (ty == (j & 15)) {
+#pragma unroll
+            for (int r = 0; r < 4; r++) {
+                if (r == rj) {
+#pragma unroll
+                    for (int c = 0; c < 8; c++) rb[tx + 8 * c] = a[r][c];
+                    if (tx == 0) rb[kMP] = bb[r];
+                }
+            }
+        }
+        if (tx == (j & 7)) {
+#pragma unroll
+            for (int c = 0; c < 8; c++) {
+                if (c == cj) {
+#pragma unroll
+                    for (int r = 0; r < 4; r++) cb[ty + 16 * r] = a[r][c];
+                }
+            }
+        }
         __syncthreads();
-        const double pj = sm.J[j * kJLD + j];
-        if (!(pj > 0.0)) { if (tid == 0) sm.scal[SC_FAIL] = 1.0; __syncthreads(); return; }
-        const double inv = rsqrt(pj);
-        double lij = 0.0;
-        if (tid > j && tid < m) { lij = sm.J[tid * kJLD + j] * inv; sm.col[tid] = lij; }
-        __syncthreads();
-        if (tid == j) sm.J[j * kJLD + j] = sqrt(pj);
-        if (tid > j && tid < m) {
-            double* row = sm.J + tid * kJLD;
-            row[j] = lij;
-            for (int l = j + 1; l <= tid; l++) row[l] = fma(-lij, sm.col[l], row[l]);
+        const double piv = rb[j];
+        if (!(piv > 0.0)) { bad = true; break; }
+        const double pinv = 1.0 / piv;
+        double rowv[8];
+#pragma unroll
+        for (int c = 0; c < 8; c++) rowv[c] = rb[tx + 8 * c];
+        const double rowb = rb[kMP];
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+            const int i = ty + 16 * r;
+            if (i == j) {
+#pragma unroll
+                for (int c = 0; c < 8; c++) a[r][c] = rowv[c] * pinv;
+                bb[r] = rowb * pinv;
+            } else {
+                const double f = cb[i] * pinv;
+#pragma unroll
+                for (int c = 0; c < 8; c++) a[r][c] = fma(-f, rowv[c], a[r][c]);
+                bb[r] = fma(-f, rowb, bb[r]);
+            }
         }
     }
-    __syncthreads();
-}
-
-// delta <- solution of L L^T delta = delta (warp 0; column-oriented substitutions)
-__device__ void fast_chol_solve(const FSm& sm, int m)
-{
-    const int tid = threadIdx.x;
-    if (tid < 32) {
-        const int lane = tid;
-        for (int i = 0; i < m; i++) {
-            if (lane == 0) sm.delta[i] = sm.delta[i] / sm.J[i * kJLD + i];
-            __syncwarp();
-            const double yi = sm.delta[i];
-            for (int l = i + 1 + lane; l < m; l += 32) sm.delta[l] = fma(-sm.J[l * kJLD + i], yi, sm.delta[l]);
-            __syncwarp();
-        }
-        for (int i = m - 1; i >= 0; i--) {
-            if (lane == 0) sm.delta[i] = sm.delta[i] / sm.J[i * kJLD + i];
-            __syncwarp();
-            const double xi = sm.delta[i];
-            for (int l = lane; l < i; l += 32) sm.delta[l] = fma(-sm.J[i * kJLD + l], xi, sm.delta[l]);
-            __syncwarp();
+    if (bad && tid == 0) sm.scal[SC_FAIL] = 1.0;
+    if (tx == 0) {
+#pragma unroll
+        for (int r = 0; r < 4; r++) {
+            const int i = ty + 16 * r;
+            if (i < m) sm.delta[i] = bb[r];
         }
     }
     __syncthreads();
@@ -455,26 +498,11 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
         rprev = rn; lam = 1.0;
         if (tid < m) sm.alpha_prev[tid] = sm.alpha[tid];
         if (tid == 0) sm.scal[SC_FAIL] = 0.0;
-        // fp64 Hessian: off-diagonal from the contraction, diagonal g - g2; an outer block's function is
-        // constant along (1,...,1): pin that direction with 1/m everywhere
-        const double add = slack ? 0.0 : 1.0 / (double)m;
-        for (int e = tid; e < m * m; e += kFT) {
-            const int i = e / m, l = e - i * m;
-            if (l <= i) {
-                const double v = (l == i) ? sm.g[i] - sm.g2[i] : -(double)sm.Jacc[i * kMP + l];
-                // (the staging area and this matrix share memory; the accumulator Jacc is separate)
-                sm.J[i * kJLD + l] = v + add;
-            }
-        }
-        __syncthreads();
-        fast_cholesky(sm, m);
+        // Newton step with the Hessian (off-diagonal from the contraction, diagonal g - g2); an outer block's
+        // function is constant along (1,...,1): pin that direction with 1/m everywhere
+        fast_newton_step(sm, m, rhs, slack ? 0.0 : 1.0 / (double)m);
         const bool fail = sm.scal[SC_FAIL] != 0.0;
-        __syncthreads();
-        if (!fail) {
-            if (tid < m) sm.delta[tid] = -(sm.g[tid] - rhs[tid]);
-            __syncthreads();
-            fast_chol_solve(sm, m);
-        } else {
+        if (fail) {
             // proportional-fitting step  alpha += log(rhs / g)
             if (tid < m) sm.delta[tid] = log(rhs[tid] / sm.g[tid]);
             __syncthreads();
