@@ -32,6 +32,7 @@ constexpr double kFTEnd = 25.0;       // quadrature range constants, identical t
 constexpr double kFDrop = 1.0;
 constexpr double kFTail = 3.0;
 constexpr int kFMaxNodes = 128;
+constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
 
@@ -51,10 +52,10 @@ struct FastLayout {
         uni = o;
         // union: staging of the Hessian operands (two float arrays [kJC][NT-1][kMP]) / elimination buffers
         const int stage_doubles = (2 * kJC * (NT - 1) * kMP * 4 + 7) / 8;
-        const int jmat_doubles = 2 * (kMP + 2) + 2 * kMP;    // pivot row / column buffers of the elimination
+        const int jmat_doubles = 2 * (kMP + 4) + 2 * kMP;    // (floats, so twice what is needed) pivot row / column buffers
         o += stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
         jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
-        o += kMP * kMP / 2;
+        o += (kMP * (kMP + 1) + 1) / 2;
         ints = o * 8;
         total_bytes = ints + KP * 3 * 4 + 64;
     }
@@ -159,7 +160,7 @@ __device__ __forceinline__ void hess_chunk(const FSm& sm, int nstaged, int m)
 #pragma unroll
     for (int a = 0; a < 4; a++)
 #pragma unroll
-        for (int b = 0; b < 8; b++) sm.Jacc[(i0 + a) * kMP + l0 + b] += acc[a][b];
+        for (int b = 0; b < 8; b++) sm.Jacc[(i0 + a) * kJS + l0 + b] += acc[a][b];
 }
 
 // g (always), and with want_jac the diagonal part g2 and the contraction Jacc, at the weights in sm.w.
@@ -178,7 +179,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
         gacc[tt] = 0.0; g2acc[tt] = 0.0;
     }
     if (want_jac) {
-        for (int e = tid; e < kMP * kMP; e += kFT) sm.Jacc[e] = 0.f;
+        for (int e = tid; e < kMP * kJS; e += kFT) sm.Jacc[e] = 0.f;
     }
     const int span = 2 * kJC;            // nodes per chunk: every second one is a Hessian node
     for (int q0 = 0; q0 < Q; q0 += span) {
@@ -337,94 +338,133 @@ __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
     __syncthreads();
 }
 
-// Newton step by Gauss-Jordan elimination without pivoting (the Hessian is symmetric positive
-// definite) on the matrix held in registers: thread (ty, tx) = (tid / 8, tid % 8) owns the entries
-// (i, l) with i = ty + 16 r, l = tx + 8 c, and the right-hand side of its rows when tx == 0.  Every
-// step publishes the pivot row and the pivot column through double-buffered shared memory, so it
-// costs one CTA barrier; after m steps the right-hand side holds the solution, with no triangular
-// substitutions.  Entries: off-diagonal -Jacc (lower triangle stored), diagonal g - g2, plus `add`
-// everywhere.  Writes the step into sm.delta; sets SC_FAIL when a pivot is not positive.
+// Newton step: fp32 Cholesky of the Hessian in place in the contraction accumulator (row stride kJS),
+// with the forward substitution carried along and the backward substitution on warp 0.  The step only
+// steers the iteration (the fp64 gradient decides convergence) and the Hessian was accumulated in fp32.
+// Thread (ty, tx) = (tid / 8, tid % 8) updates the trailing rows j+1+ty+16a and columns j+1+tx+8b.
+// Matrix: off-diagonal -Jacc (lower triangle), diagonal g - g2, plus `add` everywhere.  Writes the step
+// into sm.delta; sets SC_FAIL when a pivot is not positive.
 __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
 {
     const int tid = threadIdx.x, ty = tid >> 3, tx = tid & 7;
-    double a[4][8], bb[4];
-    double* rowbuf = sm.J;                 // [2][kMP + 2]
-    double* colbuf = sm.J + 2 * (kMP + 2); // [2][kMP]
-#pragma unroll
-    for (int r = 0; r < 4; r++) {
-        const int i = ty + 16 * r;
-#pragma unroll
-        for (int c = 0; c < 8; c++) {
-            const int l = tx + 8 * c;
-            double v;
-            if (i < m && l < m) {
-                if (i == l) v = sm.g[i] - sm.g2[i];
-                else v = -(double)(i > l ? sm.Jacc[i * kMP + l] : sm.Jacc[l * kMP + i]);
-                v += add;
-            } else {
-                v = (i == l) ? 1.0 : 0.0;
-            }
-            a[r][c] = v;
-        }
-        bb[r] = i < m ? -(sm.g[i] - rhs[i]) : 0.0;
+    float* Jm = sm.Jacc;
+    float* yv = reinterpret_cast<float*>(sm.J);        // [kMP] working right-hand side
+    float* yf = yv + kMP;                              // [kMP] forward-substituted right-hand side, then the solution
+    float* dg = yf + kMP;                              // [kMP] diagonal of the factor
+    const float addf = (float)add;
+    for (int e = tid; e < m * kMP; e += kFT) {
+        const int i = e >> 6, l = e & (kMP - 1);
+        if (l < i) Jm[i * kJS + l] = addf - Jm[i * kJS + l];
     }
-    __syncthreads();     // everyone has read Jacc / g before the buffers (which alias the staging area) are written
+    if (tid < m) {
+        Jm[tid * kJS + tid] = (float)(sm.g[tid] - sm.g2[tid]) + addf;
+        yv[tid] = -(float)(sm.g[tid] - rhs[tid]);
+    }
+    __syncthreads();
     bool bad = false;
-    for (int j = 0; j < m; j++) {
-        const int pp = j & 1;
-        double* rb = rowbuf + pp * (kMP + 2);
-        double* cb = colbuf + pp * kMP;
-        const int rj = j >> 4, cj = j >> 3;
-        if (ty == (j & 15)) {
+    // blocked right-looking factorisation, four columns per pair of barriers
+    for (int j0 = 0; j0 < m; j0 += 4) {
+        const int nb = min(4, m - j0);
+        // every thread factors the diagonal block (at most 4 x 4) in registers
+        float Lb[4][4], yb[4], dinv[4];
 #pragma unroll
-            for (int r = 0; r < 4; r++) {
-                if (r == rj) {
+        for (int c = 0; c < 4; c++) {
 #pragma unroll
-                    for (int c = 0; c < 8; c++) rb[tx + 8 * c] = a[r][c];
-                    if (tx == 0) rb[kMP] = bb[r];
-                }
+            for (int c2 = 0; c2 <= c; c2++) Lb[c][c2] = (c < nb) ? Jm[(j0 + c) * kJS + j0 + c2] : (c == c2 ? 1.f : 0.f);
+            yb[c] = (c < nb) ? yv[j0 + c] : 0.f;
+        }
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+            float dv = Lb[c][c];
+#pragma unroll
+            for (int e2 = 0; e2 < c; e2++) dv = fmaf(-Lb[c][e2], Lb[c][e2], dv);
+            if (!(dv > 0.f)) bad = true;
+            dinv[c] = rsqrtf(dv);
+            Lb[c][c] = dv * dinv[c];
+            float yc = yb[c];
+#pragma unroll
+            for (int e2 = 0; e2 < c; e2++) yc = fmaf(-Lb[c][e2], yb[e2], yc);
+            yb[c] = yc * dinv[c];
+#pragma unroll
+            for (int r2 = c + 1; r2 < 4; r2++) {
+                float v = Lb[r2][c];
+#pragma unroll
+                for (int e2 = 0; e2 < c; e2++) v = fmaf(-Lb[r2][e2], Lb[c][e2], v);
+                Lb[r2][c] = v * dinv[c];
             }
         }
-        if (tx == (j & 7)) {
+        if (bad) break;
+        __syncthreads();                       // every thread has read the block before it is overwritten
+        // panel below the block: one row per thread
+        const int i1 = j0 + nb + tid;
+        if (i1 < m) {
+            float lp[4];
+            float yi = yv[i1];
 #pragma unroll
-            for (int c = 0; c < 8; c++) {
-                if (c == cj) {
+            for (int c = 0; c < 4; c++) {
+                float v = (c < nb) ? Jm[i1 * kJS + j0 + c] : 0.f;
 #pragma unroll
-                    for (int r = 0; r < 4; r++) cb[ty + 16 * r] = a[r][c];
+                for (int e2 = 0; e2 < c; e2++) v = fmaf(-lp[e2], Lb[c][e2], v);
+                lp[c] = v * dinv[c];
+                if (c < nb) { Jm[i1 * kJS + j0 + c] = lp[c]; yi = fmaf(-lp[c], yb[c], yi); }
+            }
+            yv[i1] = yi;
+        }
+        if (tid == kFT - 1) {
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                if (c < nb) {
+                    dg[j0 + c] = Lb[c][c]; yf[j0 + c] = yb[c];
+#pragma unroll
+                    for (int c2 = 0; c2 < c; c2++) Jm[(j0 + c) * kJS + j0 + c2] = Lb[c][c2];
                 }
             }
         }
         __syncthreads();
-        const double piv = rb[j];
-        if (!(piv > 0.0)) { bad = true; break; }
-        const double pinv = 1.0 / piv;
-        double rowv[8];
+        // trailing update  J[i][l] -= sum_c L[i][c] L[l][c],  j0 + nb <= l <= i
+        const int t0 = j0 + nb;
+        float cl[8][4];
 #pragma unroll
-        for (int c = 0; c < 8; c++) rowv[c] = rb[tx + 8 * c];
-        const double rowb = rb[kMP];
+        for (int b2 = 0; b2 < 8; b2++) {
+            const int l = t0 + tx + 8 * b2;
 #pragma unroll
-        for (int r = 0; r < 4; r++) {
-            const int i = ty + 16 * r;
-            if (i == j) {
+            for (int c = 0; c < 4; c++) cl[b2][c] = (l < m && c < nb) ? Jm[l * kJS + j0 + c] : 0.f;
+        }
+        for (int i = t0 + ty; i < m; i += 16) {
+            float* row = Jm + i * kJS;
+            float ci[4];
 #pragma unroll
-                for (int c = 0; c < 8; c++) a[r][c] = rowv[c] * pinv;
-                bb[r] = rowb * pinv;
-            } else {
-                const double f = cb[i] * pinv;
+            for (int c = 0; c < 4; c++) ci[c] = (c < nb) ? row[j0 + c] : 0.f;
 #pragma unroll
-                for (int c = 0; c < 8; c++) a[r][c] = fma(-f, rowv[c], a[r][c]);
-                bb[r] = fma(-f, rowb, bb[r]);
+            for (int b2 = 0; b2 < 8; b2++) {
+                const int l = t0 + tx + 8 * b2;
+                if (l <= i) {
+                    float v = row[l];
+#pragma unroll
+                    for (int c = 0; c < 4; c++) v = fmaf(-ci[c], cl[b2][c], v);
+                    row[l] = v;
+                }
             }
         }
+        __syncthreads();
     }
-    if (bad && tid == 0) sm.scal[SC_FAIL] = 1.0;
-    if (tx == 0) {
-#pragma unroll
-        for (int r = 0; r < 4; r++) {
-            const int i = ty + 16 * r;
-            if (i < m) sm.delta[i] = bb[r];
+    if (bad) {
+        if (tid == 0) sm.scal[SC_FAIL] = 1.0;
+        __syncthreads();
+        return;
+    }
+    // backward substitution L^T x = y on warp 0 (column-oriented)
+    if (tid < 32) {
+        for (int i = m - 1; i >= 0; i--) {
+            const float xi = yf[i] / dg[i];
+            __syncwarp();
+            if (tid == 0) yf[i] = xi;
+            for (int l = tid; l < i; l += 32) yf[l] = fmaf(-Jm[i * kJS + l], xi, yf[l]);
+            __syncwarp();
         }
     }
+    __syncthreads();
+    if (tid < m) sm.delta[tid] = (double)yf[tid];
     __syncthreads();
 }
 
@@ -452,16 +492,20 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     }
     if (tid < m) sm.w[tid] = wi;
     __syncthreads();
+    // Pr[i and j drafted, all drafts inside] once, in the (still unused) contraction accumulator
+    for (int e = tid; e < m * kMP; e += kFT) {
+        const int i = e / kMP, j = e - i * kMP;
+        if (j < m) {
+            const double pij = Tn - sm.col[i] - sm.col[j] + ipow(fmax(T - d[i] - d[j], 0.0), n);
+            sm.Jacc[i * kJS + j] = (i == j) ? 0.f : (float)pij;
+        }
+    }
+    __syncthreads();
     for (int sweep = 0; sweep < 3; sweep++) {
         // S_i = sum_j Pr[i and j drafted] w_j / Pr[i drafted]: one warp per row, lanes over j
         for (int i = warp; i < m; i += kFW) {
-            const double di = d[i], zi = sm.col[i];
             double acc = 0.0;
-            for (int j = lane; j < m; j += 32) {
-                if (j == i) continue;
-                const double pij = Tn - zi - sm.col[j] + ipow(fmax(T - di - d[j], 0.0), n);
-                acc = fma(pij, sm.w[j], acc);
-            }
+            for (int j = lane; j < m; j += 32) acc = fma((double)sm.Jacc[i * kJS + j], sm.w[j], acc);
             acc = warp_sum_d(acc);
             if (lane == 0) sm.delta[i] = acc;
         }
@@ -485,9 +529,16 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     double rn = 0.0, rprev = 1.0e300, lam = 1.0;
     for (; it < max_iters; it++) {
         fast_grid(sm, m, n, slack, qstep);
-        fast_eval<NT, TPL>(sm, m, n, d, hmass, true);
+        // close to the solution the next point is expected to pass the test (quadratic convergence): evaluate
+        // the gradient alone first and add the Hessian only if the test fails after all
+        const bool expect_done = it > 0 && lam == 1.0 && rprev * rprev * 30.0 < tol;
+        fast_eval<NT, TPL>(sm, m, n, d, hmass, !expect_done);
         rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
         if (rn <= tol) { status = GR_OK; it++; break; }
+        if (expect_done) {
+            fast_eval<NT, TPL>(sm, m, n, d, hmass, true);
+            it++;
+        }
         if (!(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
             // the last step did not reduce the gradient norm: retry it at half length
             lam *= 0.5;
