@@ -32,6 +32,7 @@ constexpr double kFTEnd = 25.0;       // quadrature range constants, identical t
 constexpr double kFDrop = 1.0;
 constexpr double kFTail = 3.0;
 constexpr int kFMaxNodes = 128;
+constexpr int kMS = 72;               // row stride of the staged operands (floats): conflict-free MMA fragment loads
 constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
@@ -50,8 +51,8 @@ struct FastLayout {
         tq = o; o += kFMaxNodes; cq = o; o += kFMaxNodes;
         scal = o; o += 32;
         uni = o;
-        // union: staging of the Hessian operands (two float arrays [kJC][NT-1][kMP]) / elimination buffers
-        const int stage_doubles = (2 * kJC * (NT - 1) * kMP * 4 + 7) / 8;
+        // union: staging of the Hessian operands (two float arrays [kJC * NT][kMS]) / vectors of the Newton step
+        const int stage_doubles = (2 * kJC * NT * kMS * 4 + 7) / 8;
         const int jmat_doubles = 2 * (kMP + 4) + 2 * kMP;    // (floats, so twice what is needed) pivot row / column buffers
         o += stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
         jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
@@ -132,35 +133,74 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 
-// One chunk of the Hessian contraction: Jacc[i][l] += sum over the staged (node, kappa) of AS[.][i] HS[.][l],
-// lower triangle only.  Thread tile 4 rows x 8 columns.
+// Sum of NT-entry vectors over the 32 lanes, result in every lane.  Recursive halving: at each of the
+// first log2(NT) levels a lane keeps half of its entries and hands the other half to its partner, so the
+// exchange costs NT - 1 + (5 - log2 NT) shuffles instead of 5 NT; an all-gather of NT shuffles follows.
 template <int NT>
-__device__ __forceinline__ void hess_chunk(const FSm& sm, int nstaged, int m)
+__device__ __forceinline__ void warp_allreduce_series(double* S, int lane)
 {
-    const int tid = threadIdx.x;
-    const int i0 = (tid >> 3) * 4, l0 = (tid & 7) * 8;
-    if (i0 >= m || l0 >= m || l0 > i0 + 3) return;     // outside the matrix or wholly above the diagonal
-    float acc[4][8];
+    static_assert(NT == 4 || NT == 8, "series length");
+    int cnt = NT, o = 16;
 #pragma unroll
-    for (int a = 0; a < 4; a++)
+    for (int lvl = 0; lvl < (NT == 8 ? 3 : 2); lvl++) {
+        const int half = cnt >> 1;
+        const bool up = (lane & o) != 0;
 #pragma unroll
-        for (int b = 0; b < 8; b++) acc[a][b] = 0.f;
-    const int K = nstaged * (NT - 1);
-    for (int kk = 0; kk < K; kk++) {
-        const float4 av = *reinterpret_cast<const float4*>(sm.AS + kk * kMP + i0);
-        const float4 h0 = *reinterpret_cast<const float4*>(sm.HS + kk * kMP + l0);
-        const float4 h1 = *reinterpret_cast<const float4*>(sm.HS + kk * kMP + l0 + 4);
-        const float a4[4] = {av.x, av.y, av.z, av.w};
-        const float h8[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
-#pragma unroll
-        for (int a = 0; a < 4; a++)
-#pragma unroll
-            for (int b = 0; b < 8; b++) acc[a][b] = fmaf(a4[a], h8[b], acc[a][b]);
+        for (int c = 0; c < NT / 2; c++) {
+            if (c < half) {
+                const double keep = up ? S[c + half] : S[c];
+                const double send = up ? S[c] : S[c + half];
+                S[c] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
+        }
+        cnt = half; o >>= 1;
     }
+    double v = S[0];
+    for (; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    // lane bits (4, 3[, 2]) say which entry the lane holds
 #pragma unroll
-    for (int a = 0; a < 4; a++)
-#pragma unroll
-        for (int b = 0; b < 8; b++) sm.Jacc[(i0 + a) * kJS + l0 + b] += acc[a][b];
+    for (int c = 0; c < NT; c++) {
+        const int src = (NT == 8) ? ((((c >> 2) & 1) << 4) | (((c >> 1) & 1) << 3) | ((c & 1) << 2))
+                                  : ((((c >> 1) & 1) << 4) | ((c & 1) << 3));
+        S[c] = __shfl_sync(0xffffffffu, v, src);
+    }
+}
+
+// tf32 rounding of a staged operand (the contraction runs on the tensor cores: it is the one dense
+// contraction of the path, and it only steers Newton's method)
+__device__ __forceinline__ float to_tf32(float x) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return __uint_as_float(u);
+}
+
+// One chunk of the Hessian contraction: Jacc[i][l] += sum over the staged rows kk of AS[kk][i] HS[kk][l] for the
+// 16 x 8 tiles that touch the lower triangle, as m16n8k8 tf32 MMAs with fp32 accumulation.  K8 = staged rows,
+// a multiple of 8.  The 20 lower tiles of the 64 x 64 matrix are dealt round-robin to the four warps.
+__device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    for (int t = warp; t < 20; t += kFW) {
+        const int mi = t >= 12 ? 3 : (t >= 6 ? 2 : (t >= 2 ? 1 : 0));
+        const int ni = t - (mi == 3 ? 12 : (mi == 2 ? 6 : (mi == 1 ? 2 : 0)));
+        const int i0 = 16 * mi, l0 = 8 * ni;
+        if (i0 >= m || l0 >= m) continue;
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+        for (int k0 = 0; k0 < K8; k0 += 8) {
+            const float* Ap = sm.AS + (k0 + tig) * kMS + i0 + gid;
+            const float* Bp = sm.HS + (k0 + tig) * kMS + l0 + gid;
+            const uint32_t a0 = __float_as_uint(Ap[0]), a1 = __float_as_uint(Ap[8]);
+            const uint32_t a2 = __float_as_uint(Ap[4 * kMS]), a3 = __float_as_uint(Ap[4 * kMS + 8]);
+            const uint32_t b0 = __float_as_uint(Bp[0]), b1 = __float_as_uint(Bp[4 * kMS]);
+            asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                         : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+                         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        }
+        float* J0 = sm.Jacc + (i0 + gid) * kJS + l0 + 2 * tig;
+        J0[0] += c0; J0[1] += c1;
+        J0[8 * kJS] += c2; J0[8 * kJS + 1] += c3;
+    }
 }
 
 // g (always), and with want_jac the diagonal part g2 and the contraction Jacc, at the weights in sm.w.
@@ -207,11 +247,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
                 }
             }
             // log-derivative of the product: sum over the tokens (all lanes end with the totals)
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-                for (int c = 0; c < NT; c++) S[c] += __shfl_xor_sync(0xffffffffu, S[c], o);
-            }
+            warp_allreduce_series<NT>(S, lane);
             S[0] += hmass;
             // P' = S P, column-oriented
             double P[NT + 1], acc[NT + 1];
@@ -278,20 +314,31 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
                             }
                         }
                         const bool live = kap < n;
-                        sm.AS[(slot * (NT - 1) + kap - 1) * kMP + j] = live ? (float)(sa * a) : 0.f;
-                        sm.HS[(slot * (NT - 1) + kap - 1) * kMP + j] = live ? (float)(u * hd[kap]) : 0.f;
-                        if (TPL == 1) {
-                            sm.AS[(slot * (NT - 1) + kap - 1) * kMP + j + 32] = 0.f;
-                            sm.HS[(slot * (NT - 1) + kap - 1) * kMP + j + 32] = 0.f;
-                        }
+                        const int row = slot * NT + kap - 1;
+                        sm.AS[row * kMS + j] = live ? to_tf32((float)(sa * a)) : 0.f;
+                        sm.HS[row * kMS + j] = live ? to_tf32((float)(u * hd[kap])) : 0.f;
+                        if (TPL == 1) { sm.AS[row * kMS + j + 32] = 0.f; sm.HS[row * kMS + j + 32] = 0.f; }
+                    }
+                    // the NT-th row of the node's slot pads the contraction length to a multiple of the MMA depth
+                    sm.AS[(slot * NT + NT - 1) * kMS + j] = 0.f;
+                    sm.HS[(slot * NT + NT - 1) * kMS + j] = 0.f;
+                    if (TPL == 1) {
+                        sm.AS[(slot * NT + NT - 1) * kMS + j + 32] = 0.f;
+                        sm.HS[(slot * NT + NT - 1) * kMS + j + 32] = 0.f;
                     }
                 }
             }
         }
         if (want_jac) {
-            __syncthreads();
             const int nstaged = (q1 - q0 + 1) >> 1;
-            hess_chunk<NT>(sm, nstaged, m);
+            int K8 = nstaged * NT;
+            if (K8 & 7) {
+                // NT = 4 with an odd number of staged nodes: one more all-zero slot completes the MMA depth
+                for (int e = tid; e < NT * kMS; e += kFT) { sm.AS[K8 * kMS + e] = 0.f; sm.HS[K8 * kMS + e] = 0.f; }
+                K8 += NT;
+            }
+            __syncthreads();
+            hess_chunk(sm, K8, m);
             __syncthreads();
         }
     }
@@ -453,13 +500,33 @@ __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double
         __syncthreads();
         return;
     }
-    // backward substitution L^T x = y on warp 0 (column-oriented)
+    // backward substitution L^T x = y on warp 0, four unknowns at a time: every lane solves the 4 x 4
+    // triangle redundantly, then the lanes update the unknowns above it
     if (tid < 32) {
-        for (int i = m - 1; i >= 0; i--) {
-            const float xi = yf[i] / dg[i];
+        for (int e0 = ((m - 1) >> 2) << 2; e0 >= 0; e0 -= 4) {
+            const int nb = min(4, m - e0);
+            float x[4];
+#pragma unroll
+            for (int c = 3; c >= 0; c--) {
+                float v = 0.f;
+                if (c < nb) {
+                    v = yf[e0 + c];
+#pragma unroll
+                    for (int c2 = 3; c2 > c; c2--)
+                        if (c2 < nb) v = fmaf(-Jm[(e0 + c2) * kJS + e0 + c], x[c2], v);
+                    v = v / dg[e0 + c];
+                }
+                x[c] = v;
+            }
             __syncwarp();
-            if (tid == 0) yf[i] = xi;
-            for (int l = tid; l < i; l += 32) yf[l] = fmaf(-Jm[i * kJS + l], xi, yf[l]);
+            if (tid < nb) yf[e0 + tid] = tid == 0 ? x[0] : (tid == 1 ? x[1] : (tid == 2 ? x[2] : x[3]));
+            for (int l = tid; l < e0; l += 32) {
+                float v = yf[l];
+#pragma unroll
+                for (int c = 0; c < 4; c++)
+                    if (c < nb) v = fmaf(-Jm[(e0 + c) * kJS + l], x[c], v);
+                yf[l] = v;
+            }
             __syncwarp();
         }
     }
@@ -602,7 +669,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     sm.gw = base + L.gw; sm.g2w = base + L.g2w; sm.tq = base + L.tq; sm.cq = base + L.cq; sm.scal = base + L.scal;
     sm.J = base + L.uni;
     sm.AS = reinterpret_cast<float*>(base + L.uni);
-    sm.HS = sm.AS + kJC * (NT - 1) * kMP;
+    sm.HS = sm.AS + kJC * NT * kMS;
     sm.Jacc = reinterpret_cast<float*>(smem_raw + L.jacc_bytes_off);
     int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
     sm.id = ib; sm.blk = ib + KP; sm.itmp = ib + 2 * KP;
