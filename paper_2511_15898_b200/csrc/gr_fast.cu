@@ -364,8 +364,19 @@ __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
     double* red = sm.scal + SC_RED;
     double a = 0.0;
     if (tid < m) { a = sm.alpha[tid]; sm.w[tid] = exp(a); }
-    const double hi = block_reduce_max(tid < m ? a : -1.0e300, red);
-    const double lo = -block_reduce_max(tid < m ? -a : -1.0e300, red);
+    // extreme alphas in one pass (they give the extreme weights)
+    double hi = tid < m ? a : -1.0e300, lo = tid < m ? -a : -1.0e300;
+    for (int o = 16; o > 0; o >>= 1) {
+        hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        lo = fmax(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    }
+    __syncthreads();
+    if ((tid & 31) == 0) { red[2 * (tid >> 5)] = hi; red[2 * (tid >> 5) + 1] = lo; }
+    __syncthreads();
+    hi = red[0]; lo = red[1];
+#pragma unroll
+    for (int i = 1; i < kFW; i++) { hi = fmax(hi, red[2 * i]); lo = fmax(lo, red[2 * i + 1]); }
+    lo = -lo;
     const double wmax = exp(hi), wmin = exp(lo);
     const double rate = slack ? 1.0 + wmin : wmin;
     const double s_hi = log(kFTEnd / rate);
