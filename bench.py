@@ -30,6 +30,9 @@ METRIC = "solve+verify instances/sec at V=128256,n=8,top-k=50"
 UNIT = "instances/s"
 HEADLINE = dict(V=128256, n=8, topk=50, batch=1024, temp_target=0.7, temp_draft=1.0)
 BYTES_PER_INSTANCE = HEADLINE["V"] * (4 + 4)       # both fp32 logit rows, read once
+# dram__bytes_read + dram__bytes_write of scan_kernel per instance, from the ncu capture at batch 296
+# (profiles/scan_kernel_config3_batch296.md); traffic is proportional to the rows read
+SCAN_TRAFFIC_PER_INSTANCE = (304.640256e6 + 4.621056e6) / 296
 
 
 def _peaks():
@@ -55,7 +58,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -244,13 +247,28 @@ def run_ours(args):
     solve_avg_ms = float(np.mean(solve_ms))
     ach = BYTES_PER_INSTANCE * B / (scan_avg_ms * 1e-3) / 1e9
     path_gbs = BYTES_PER_INSTANCE * B / (float(np.mean(step_ms)) * 1e-3) / 1e9
+    # dominant kernel: the solve kernel (fp64 arithmetic).  Algorithmic FMAs per gradient evaluation = nodes x
+    # [k (n(n-1)/2 + 2n) + n(n+1)/2] (series of every token, log-derivative sum, product recurrence, extraction),
+    # nodes = 26 at this shape; evaluations per instance are read back from the rule.
+    rule = G.read_rule(solved)
+    evals = float(rule.iters.float().mean().item())
+    n_, k_ = H["n"], H["topk"]
+    fma_eval = 26 * (k_ * (n_ * (n_ - 1) // 2 + 2 * n_) + n_ * (n_ + 1) // 2)
+    flops = 2.0 * fma_eval * evals * B
+    solve_kernel_ms = solve_avg_ms - scan_avg_ms
+    ach_tf = flops / (solve_kernel_ms * 1e-3) / 1e12
+    fp64_peak = 148 * 64 * 2 * 1.965e9 / 1e12      # SMs x fp64 FMA lanes x 2 x max SM clock
+    roof = {"bound": "alu", "kernel": "fast_solve_kernel (fp64 Newton solve; dominant)", "achieved": ach_tf,
+            "peak": fp64_peak, "unit": "TFLOP/s", "frac": ach_tf / fp64_peak, "traffic": None,
+            "peak_kind": "derived: 148 SMs x 64 fp64 FMA/clk x 1.965 GHz", "kernel_ms": solve_kernel_ms,
+            "evals_per_instance": evals}
     status = solved.status.cpu().numpy()
     acc_rate = float(ver.accepted.float().mean().item())
 
     # ---- batch-1 call latency
     wl1 = wl.rows([0])
     s1 = None; v1 = None
-    lat = [float("nan")]
+    lat = []
     for i in range(0 if args.no_extras else 30):
         a = torch.cuda.Event(enable_timing=True); b_ = torch.cuda.Event(enable_timing=True)
         a.record()
@@ -281,16 +299,19 @@ def run_ours(args):
         "config": {"workload": f"config3: V=128256 n=8 top-k=50 batch {B} per GPU, fp32 logits, target temp 0.7, "
                                "draft temp 1.0, Zipf-shaped logits", "global_batch": world * B,
                    "cache": f"inputs ({BYTES_PER_INSTANCE * B / 1e9:.2f} GB per batch) larger than L2, no flush needed", "parallelism": f"batch x{world}"},
-        "roofline": {"bound": "hbm", "kernel": "scan_kernel (streams both logit rows once)", "achieved": ach,
-                     "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": None, "peak_kind": peak_kind,
-                     "kernel_ms": scan_avg_ms, "path_achieved": path_gbs, "path_frac": path_gbs / peak},
+        "roofline": roof,
+        "roofline_scan": {"bound": "hbm", "kernel": "scan_kernel (streams both logit rows once)", "achieved": ach,
+                          "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": SCAN_TRAFFIC_PER_INSTANCE * B,
+                          "peak_kind": peak_kind, "kernel_ms": scan_avg_ms},
+        "roofline_path": {"bound": "hbm", "what": "bytes of both logit rows / whole solve+verify step time",
+                          "achieved": path_gbs, "peak": peak, "unit": "GB/s", "frac": path_gbs / peak},
         "kernels_ms": {"scan": scan_avg_ms, "solve": solve_avg_ms - scan_avg_ms, "verify": float(np.mean(verify_ms))},
         "p50_us": {"batch_step": float(np.median(step_ms)) * 1e3,
                    "per_instance_amortised": float(np.median(step_ms)) * 1e3 / B,
-                   "batch1_call": float(np.median(lat))},
+                   "batch1_call": float(np.median(lat)) if lat else None},
         "cpu_baseline": cpu,
         "e2e": e2e,
-        "gpu_launches": 3 * K,
+        "gpu_launches": 4 * K,   # scan, fast solve, robust solve (flagged instances only), verify
         "clocks": clocks,
         "quality": {"accept_rate": acc_rate, "status_ok": int((status == 0).sum()),
                     "status_not_converged": int((status == 1).sum()), "wall_ms_total": total_ms},
@@ -303,8 +324,8 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=HEADLINE["batch"],
                     help="instances per GPU (default: the headline 1024; smaller values are for profiler captures)")
