@@ -19,7 +19,7 @@
 
 namespace gr {
 
-constexpr int kScanThreads = 1024;
+constexpr int kScanThreads = 512;    // two CTAs per SM: one CTA's epilogue overlaps the other's streaming
 constexpr int kScanWarps = kScanThreads / 32;
 constexpr int kCandCap = 2048;
 constexpr int kMaxChunks = 2049;     // V <= 2^21
@@ -153,7 +153,7 @@ __device__ void exact_select_slow(const T* prow, int V, int ksel, const CandList
 // kFull: the support is the whole vocabulary and exceeds kMaxSupport; no support is
 // selected, the draft row's log-sum-exp is produced instead.
 template <typename T, bool kFull>
-__global__ void __launch_bounds__(kScanThreads, 1)
+__global__ void __launch_bounds__(kScanThreads, 2)
 scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, float sc_t, float sc_d,
             double temp_t, double temp_d, char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap)
 {
@@ -333,28 +333,38 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
         }
         if (M > kCandCap) M = kCandCap;
         // composite keys in place of the (value, id) pairs
-        float v0 = 0.f, v1 = 0.f; int i0 = 0, i1 = 0;
-        if (tid < M) { v0 = cl.v[tid]; i0 = cl.id[tid]; }
-        if (tid + kScanThreads < M) { v1 = cl.v[tid + kScanThreads]; i1 = cl.id[tid + kScanThreads]; }
+        constexpr int kPer = kCandCap / kScanThreads;
+        float vv[kPer]; int ii[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; u++) {
+            const int e = tid + u * kScanThreads;
+            vv[u] = 0.f; ii[u] = 0;
+            if (e < M) { vv[u] = cl.v[e]; ii[u] = cl.id[e]; }
+        }
         __syncthreads();
-        if (tid < M) s_keys[tid] = ckey(v0, i0);
-        if (tid + kScanThreads < M) s_keys[tid + kScanThreads] = ckey(v1, i1);
+#pragma unroll
+        for (int u = 0; u < kPer; u++) {
+            const int e = tid + u * kScanThreads;
+            if (e < M) s_keys[e] = ckey(vv[u], ii[u]);
+        }
         __syncthreads();
         char* wsb = ws + (size_t)b * ws_stride();
         int* w_id = reinterpret_cast<int*>(wsb + sizeof(WsHeader));
         float* w_dl = reinterpret_cast<float*>(w_id + kMaxSupport);
         float* w_tl = w_dl + kMaxSupport;
         if (M < nsel) nsel = M;   // cannot happen for finite rows; keeps the writes in range
-        for (int e = tid; e < M; e += kScanThreads) {
-            const unsigned long long me = s_keys[e];
-            int rank = 0;
-            for (int j = 0; j < M; j++) rank += (s_keys[j] > me) ? 1 : 0;
-            if (rank < nsel) {
-                float v = e < kScanThreads ? v0 : v1;
-                int id = e < kScanThreads ? i0 : i1;
-                w_id[rank] = id;
-                w_dl[rank] = v;
-                w_tl[rank] = load_logit<T>(qrow, id);
+#pragma unroll
+        for (int u = 0; u < kPer; u++) {
+            const int e = tid + u * kScanThreads;
+            if (e < M) {
+                const unsigned long long me = s_keys[e];
+                int rank = 0;
+                for (int j = 0; j < M; j++) rank += (s_keys[j] > me) ? 1 : 0;
+                if (rank < nsel) {
+                    w_id[rank] = ii[u];
+                    w_dl[rank] = vv[u];
+                    w_tl[rank] = load_logit<T>(qrow, ii[u]);
+                }
             }
         }
     }
