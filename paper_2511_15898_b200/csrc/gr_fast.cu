@@ -204,9 +204,10 @@ __device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
 }
 
 // g (always), and with want_jac the diagonal part g2 and the contraction Jacc, at the weights in sm.w.
+// The contraction takes every jstride-th node (weights scaled by jstride).
 // Node abscissae / weights are in sm.tq / sm.cq, their number in sm.scal[SC_Q].
 template <int NT, int TPL>
-__device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double hmass, bool want_jac)
+__device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double hmass, bool want_jac, int jstride)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, KP = sm.KP;
     const int Q = (int)sm.scal[SC_Q];
@@ -221,7 +222,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
     if (want_jac) {
         for (int e = tid; e < kMP * kJS; e += kFT) sm.Jacc[e] = 0.f;
     }
-    const int span = 2 * kJC;            // nodes per chunk: every second one is a Hessian node
+    const int span = jstride * kJC;      // nodes per chunk: every jstride-th one is a Hessian node
     for (int q0 = 0; q0 < Q; q0 += span) {
         const int q1 = min(Q, q0 + span);
         for (int q = q0 + warp; q < q1; q += kFW) {
@@ -275,8 +276,8 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
                 }
             }
             const double cq = sm.cq[q];
-            const bool jnode = want_jac && ((q & 1) == 0);
-            const int slot = (q - q0) >> 1;
+            const bool jnode = want_jac && ((q - q0) % jstride == 0);
+            const int slot = (q - q0) / jstride;
 #pragma unroll
             for (int tt = 0; tt < TPL; tt++) {
                 double hh[NT + 1], hd[NT + 1];
@@ -297,7 +298,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
                     // A = P h (series), paired as  sum_kappa A[n - kappa] h_l[kappa],  kappa = 1..n-1.
                     // Staged scaled: AS = 2 c_q t u A[n - kappa] (the 2: every second node), HS = u h[kappa].
                     const int j = lane + 32 * tt;
-                    const double sa = 2.0 * cq * t * u;
+                    const double sa = (double)jstride * cq * t * u;
 #pragma unroll
                     for (int kap = 1; kap < NT; kap++) {
                         double a = 0.0;                  // A[e], e = n - kap, = sum_{c=1..e} h[c] P[e - c]
@@ -330,7 +331,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
             }
         }
         if (want_jac) {
-            const int nstaged = (q1 - q0 + 1) >> 1;
+            const int nstaged = (q1 - q0 + jstride - 1) / jstride;
             int K8 = nstaged * NT;
             if (K8 & 7) {
                 // NT = 4 with an odd number of staged nodes: one more all-zero slot completes the MMA depth
@@ -606,15 +607,19 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     int status = GR_NOT_CONVERGED, it = 0;
     double rn = 0.0, rprev = 1.0e300, lam = 1.0;
     for (; it < max_iters; it++) {
-        fast_grid(sm, m, n, slack, qstep);
+        // far from the solution the trapezoid step is doubled (quadrature error ~4e-6, far below the gradient
+        // norm there): half the nodes, every one of them a Hessian node.  Convergence is only ever declared on
+        // the full grid.
+        const bool coarse = rprev > 1.0e-2;
+        fast_grid(sm, m, n, slack, coarse ? 2.0 * qstep : qstep);
         // close to the solution the next point is expected to pass the test (quadratic convergence): evaluate
         // the gradient alone first and add the Hessian only if the test fails after all
-        const bool expect_done = it > 0 && lam == 1.0 && rprev * rprev * 30.0 < tol;
-        fast_eval<NT, TPL>(sm, m, n, d, hmass, !expect_done);
+        const bool expect_done = !coarse && it > 0 && lam == 1.0 && rprev * rprev * 30.0 < tol;
+        fast_eval<NT, TPL>(sm, m, n, d, hmass, !expect_done, coarse ? 1 : 2);
         rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
-        if (rn <= tol) { status = GR_OK; it++; break; }
+        if (rn <= tol && !coarse) { status = GR_OK; it++; break; }
         if (expect_done) {
-            fast_eval<NT, TPL>(sm, m, n, d, hmass, true);
+            fast_eval<NT, TPL>(sm, m, n, d, hmass, true, 2);
             it++;
         }
         if (!(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
