@@ -36,6 +36,7 @@ constexpr int kMS = 72;               // row stride of the staged operands (floa
 constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
+constexpr int kFSweeps = 3;           // fixed-point sweeps of the mean-field start
 
 struct FastLayout {
     int KP;
@@ -580,13 +581,24 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
         }
     }
     __syncthreads();
-    for (int sweep = 0; sweep < 3; sweep++) {
-        // S_i = sum_j Pr[i and j drafted] w_j / Pr[i drafted]: one warp per row, lanes over j
-        for (int i = warp; i < m; i += kFW) {
-            double acc = 0.0;
-            for (int j = lane; j < m; j += 32) acc = fma((double)sm.Jacc[i * kJS + j], sm.w[j], acc);
-            acc = warp_sum_d(acc);
-            if (lane == 0) sm.delta[i] = acc;
+    for (int sweep = 0; sweep < kFSweeps; sweep++) {
+        // S_i = sum_j Pr[i and j drafted] w_j / Pr[i drafted]: four rows per warp at a time (independent
+        // reductions interleave), lanes over j
+        for (int i0 = 4 * warp; i0 < m; i0 += 4 * kFW) {
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int j = lane; j < m; j += 32) {
+                const double wj = sm.w[j];
+#pragma unroll
+                for (int a2 = 0; a2 < 4; a2++)
+                    if (i0 + a2 < m) acc[a2] = fma((double)sm.Jacc[(i0 + a2) * kJS + j], wj, acc[a2]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int a2 = 0; a2 < 4; a2++) acc[a2] += __shfl_xor_sync(0xffffffffu, acc[a2], o);
+            }
+            if (lane < 4 && i0 + lane < m)
+                sm.delta[i0 + lane] = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
         }
         __syncthreads();
         if (tid < m) {
