@@ -137,6 +137,7 @@ def run_ours(args):
     import paper_2511_15898_b200 as G
     from paper_2511_15898_b200 import workloads as W
     from paper_2511_15898_b200.build import build_library
+    from paper_2511_15898_b200.sharding import max_over_ranks
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -205,11 +206,7 @@ def run_ours(args):
     verify_ms = [e[1].elapsed_time(e[2]) for e in evs]
     step_ms = [e[0].elapsed_time(e[2]) for e in evs]
     # the per-step sync above adds host gaps between steps; the step time is the device time of the two calls
-    dev_ms = float(np.sum(step_ms))
-    t = torch.tensor([dev_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dev_ms = float(t.item())
+    dev_ms = max_over_ranks(float(np.sum(step_ms)), dev)      # slowest rank's device time
     value = world * B * K / (dev_ms * 1e-3)
 
     # ---- end to end through the public API with host (pinned) buffers
@@ -228,12 +225,10 @@ def run_ours(args):
                                                    None, dev, state)
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        te = torch.tensor([dt], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        dt_max = max_over_ranks(dt, dev)
         h2d = hq.numel() * hq.element_size() * 2 + ht.numel() * 4 + hu.numel() * 4
         d2h = B * (4 + 1 + 4 + 4)
-        e2e = {"value": world * B * Ke / float(te.item()), "unit": UNIT, "h2d_bytes_per_step": int(h2d),
+        e2e = {"value": world * B * Ke / dt_max, "unit": UNIT, "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "steps": Ke}
         del hq, hp
 

@@ -369,3 +369,15 @@ def test_draft_token_outside_support_is_an_error():
     outside = [i for i in range(10) if i not in sol.order.tolist()][0]
     nu, *_ = O.slice_(sol, [int(sol.order[0]), outside])
     assert nu == O.GRO_DRAFT_OUT_OF_SUPPORT
+
+
+def test_golden_config1_values_have_not_drifted():
+    """tests/golden/config1_oracle.txt was written by tests/golden/make_golden.py from the oracle alone."""
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "config1_oracle.txt")
+    rows = [ln.split() for ln in open(path) if not ln.startswith("#")]
+    wl = W.config1(batch=8)
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    for b, a, js, nb in rows:
+        sol = O.solve(tl[int(b)], dl[int(b)], wl.n, wl.topk, tol=1e-12)
+        assert abs(sol.alpha_star - float(a)) < 1e-13 and sol.jstar == int(js) and sol.nblocks == int(nb)
