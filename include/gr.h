@@ -118,7 +118,8 @@ size_t gr_workspace_bytes(int V, int n, int topk, int batch);
  *                       so q_logits must stay unchanged until gr_verify has run.
  *   workspace           scratch, gr_workspace_bytes() bytes, 16-byte aligned;
  *                       contents are meaningless after the call completes.
- *   alpha_star          out [batch] float, optimal acceptance probability.
+ *   alpha_star          out [batch] float, optimal acceptance probability (also produced, by a sort of
+ *                       the whole row, when the support exceeds GR_MAX_SUPPORT and no rule is solved).
  *   status              out [batch] int, GR_OK / GR_NOT_CONVERGED /
  *                       GR_SUPPORT_TOO_LARGE / GR_BAD_LOGITS.
  */
@@ -139,6 +140,8 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
  * The scratch is a fixed array inside the library's device image, GR_STATIC_MAX_BATCH
  * instances large (about 0.4 MB, held by every GPU that loads the library until exit).
  *   - batch > GR_STATIC_MAX_BATCH returns GR_E_TOO_LARGE and launches nothing; split the batch.
+ *     So does an untruncated draft on a vocabulary larger than GR_MAX_SUPPORT (its alpha* needs a
+ *     per-row sort buffer the built-in scratch does not have).
  *   - The first call on each device looks the array's device address up (that device must
  *     be current, as for any launch); make that first call before any stream capture.
  *   - The call itself allocates and frees nothing.

@@ -60,6 +60,24 @@ def distributions(tl, dl, topk, Tt, Td):
     return tgt, drf, ids[:k].copy(), lse.value
 
 
+def alpha_star_only(tl, dl, n, topk, Tt=1.0, Td=1.0):
+    """Optimal acceptance and |H*| alone (distributions + subset selection, no convex solve): usable on
+    supports far too large for the solvers."""
+    tl, dl = _f64(tl), _f64(dl)
+    V = tl.shape[0]
+    tgt, drf, ids, _ = distributions(tl, dl, topk, Tt, Td)
+    k = ids.shape[0]
+    ids = _i32(ids)
+    order = np.empty(k, dtype=np.int32)
+    psi = np.empty(k + 1); Tg = np.empty(k + 1); Dr = np.empty(k + 1)
+    a = C.c_double(0)
+    D = C.c_double
+    js = lib().gro_subset_selection(_p(tl, D), _p(dl, D), _p(tgt, D), _p(drf, D), _p(ids, C.c_int), k, int(n),
+                                    D(Tt), D(Td), int(k == V), _p(order, C.c_int), _p(psi, D), _p(Tg, D), _p(Dr, D),
+                                    C.byref(a))
+    return a.value, int(js)
+
+
 def grad(route, d, w, n, h=0.0, slack=True):
     d, w = _f64(d), _f64(w)
     m = d.shape[0]

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgr_b200.so")
-SOURCES = ["gr_api.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_verify.cu"]
+SOURCES = ["gr_api.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_fullsort.cu", "gr_verify.cu"]
 HEADERS = [os.path.join(CSRC, "gr_common.cuh"), os.path.join(CSRC, "gr_prep.cuh"), os.path.join(ROOT, "include", "gr.h")]
 
 

@@ -11,6 +11,9 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
 int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
                 cudaStream_t st);
+size_t fullsort_scratch_bytes(int V);
+void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
+                     const char* ws, char* scratch, char* params, int pstride, float* alpha_out, cudaStream_t st);
 void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
                    unsigned char* out_acc, int* status, cudaStream_t st);
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
@@ -48,8 +51,11 @@ size_t gr_params_bytes(int V, int n, int topk, int batch)
 size_t gr_workspace_bytes(int V, int n, int topk, int batch)
 {
     if (!gr::shape_ok(V, n, batch)) return 0;
-    (void)topk;
-    return (size_t)gr::ws_stride() * (size_t)(batch > 0 ? batch : 1);
+    const size_t nb = (size_t)(batch > 0 ? batch : 1);
+    size_t s = (size_t)gr::ws_stride() * nb;
+    // an untruncated draft on a vocabulary beyond the solve capacity: room to sort the row for alpha*
+    if (gr::kcap_of(V, topk) == 0) s += gr::fullsort_scratch_bytes(V) * nb;
+    return s;
 }
 
 int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
@@ -89,6 +95,12 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
                                   (double)temp_target, (double)temp_draft, tol, max_iters, qstep, batch, force_robust,
                                   alpha_star, status, st);
     if (rc != GR_OK) return rc;
+    if (full_large) {
+        // no rule is solved for this shape, but the optimal acceptance still is (sort + prefix scan)
+        char* scratch = (char*)workspace + (size_t)gr::ws_stride() * (size_t)batch;
+        gr::launch_fullsort(q_logits, p_logits, dtype, V, n, (double)temp_target, (double)temp_draft, batch,
+                            (const char*)workspace, scratch, (char*)params, pstride, alpha_star, st);
+    }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;
 }

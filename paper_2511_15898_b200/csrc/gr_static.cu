@@ -64,7 +64,7 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     const int kfull = (topk <= 0 || topk >= V) ? V : topk;
     const int kcap = gr::kcap_of(V, topk);
     const bool full_large = kcap == 0;
-    if (full_large && kfull != V) return GR_E_TOO_LARGE;
+    if (full_large) return GR_E_TOO_LARGE;     // (the built-in scratch has no room for the whole-vocabulary sort)
     char* ws = nullptr;
     const int rs = gr::static_workspace(&ws);
     if (rs != GR_OK) return rs;

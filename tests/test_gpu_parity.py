@@ -122,6 +122,12 @@ def test_support_beyond_capacity_falls_back_to_target_sampling():
     ver = G.verify(solved, wl.draft_tokens, wl.uniforms)
     torch.cuda.synchronize()
     assert solved.status.cpu().tolist() == [G.GR_SUPPORT_TOO_LARGE] * 6
+    # the optimal acceptance is still produced (whole-row sort + prefix scan)
+    from oracle import gr_oracle as O
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    for b in range(6):
+        a, _ = O.alpha_star_only(tl[b], dl[b], wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+        assert abs(float(solved.alpha_star[b]) - a) <= ALPHA_TOL
     tgt = torch.softmax(wl.q_logits.double(), dim=1).cpu().numpy()
     u1 = wl.uniforms[:, 1].double().cpu().numpy()
     tok = ver.token.cpu().numpy(); acc = ver.accepted.cpu().numpy()
@@ -167,3 +173,19 @@ def test_host_buffer_front_end_matches_device_front_end():
     tok, acc, al, st = G.solve_verify_host(wl.q_logits.cpu(), wl.p_logits.cpu(), wl.draft_tokens.cpu(),
                                            wl.uniforms.cpu(), wl.n, wl.topk)
     assert torch.equal(tok, v.token.cpu()) and torch.equal(al, s.alpha_star.cpu())
+
+
+@pytest.mark.parametrize("n,sigma", [(2, 0.25), (8, 1.0), (32, 2.0)])
+def test_config4_whole_vocabulary_cells_alpha_star(n, sigma):
+    """k = V = 50257: no rule on the GPU (and none the oracle could solve either), but alpha* must match."""
+    from oracle import gr_oracle as O
+    wl = W.config4(n, 0, sigma, batch=4, device="cuda")
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+    ver = G.verify(solved, wl.draft_tokens, wl.uniforms)
+    torch.cuda.synchronize()
+    assert solved.status.cpu().tolist() == [G.GR_SUPPORT_TOO_LARGE] * 4
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    for b in range(4):
+        a, _ = O.alpha_star_only(tl[b], dl[b], wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+        assert abs(float(solved.alpha_star[b]) - a) <= ALPHA_TOL, (b, float(solved.alpha_star[b]), a)
+    assert bool((ver.token >= 0).all())

@@ -381,3 +381,14 @@ def test_golden_config1_values_have_not_drifted():
     for b, a, js, nb in rows:
         sol = O.solve(tl[int(b)], dl[int(b)], wl.n, wl.topk, tol=1e-12)
         assert abs(sol.alpha_star - float(a)) < 1e-13 and sol.jstar == int(js) and sol.nblocks == int(nb)
+
+
+def test_alpha_star_only_agrees_with_the_full_solve_and_with_enumeration():
+    rng = np.random.default_rng(314)
+    for V, n, topk in [(10, 3, 0), (12, 2, 5), (9, 8, 0)]:
+        tl, dl = _rand_logits(rng, V)
+        a, js = O.alpha_star_only(tl, dl, n, topk)
+        sol = O.solve(tl, dl, n, topk, tol=1e-6, max_iter=5)
+        assert a == sol.alpha_star and js == sol.jstar
+        tgt, drf, _, _ = O.distributions(tl, dl, topk, 1.0, 1.0)
+        assert abs(a - (1.0 + BF.all_subset_psi(tgt, drf, n).min())) < 1e-13
