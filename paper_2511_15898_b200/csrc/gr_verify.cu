@@ -24,27 +24,16 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
 // Two levels: per-chunk masses from the scan kernel's table minus the flow p_i of the
 // support ids in the chunk, then an exact fp64 pass over the one chunk selected.
 __device__ int resample_draw(const Header* h, const ParamView& pv, int k, double frac, int lane,
-                             int* l_id, double* l_r)
+                             int* l_id, double* l_r, int* s_id, double* s_p)
 {
     const int nch = h->nch, head = h->head, V = h->V, dtype = h->dtype;
     const double T = (double)h->temp_target, lse = h->lse_t;
     const void* row = h->q_row;
-    // chunk masses, 32 at a time
-    double total = 0.0;
-    for (int c0 = 0; c0 < nch; c0 += 32) {
-        const int c = c0 + lane;
-        double R = 0.0;
-        if (c < nch) {
-            const float2 ms = pv.chunk[c];
-            R = (double)ms.y * exp((double)ms.x / T - lse);
-            const int cb = chunk_begin(c, head), ce = chunk_end(c, head, nch, V);
-            for (int j = 0; j < k; j++) { const int id = pv.id[j]; if (id >= cb && id < ce) R -= pv.p[j]; }
-            if (R < 0.0) R = 0.0;
-        }
-        total += R;
-    }
-    total = warp_sum(total);
-    const double thr = frac * total;
+    // The total residual mass is known in closed form (1 - alpha*, or 1 when the target itself is sampled), so
+    // one pass over the chunk masses finds the chunk.  The support's (id, flow) pairs are staged in shared memory.
+    for (int j = lane; j < k; j += 32) { s_id[j] = pv.id[j]; s_p[j] = pv.p[j]; }
+    __syncwarp();
+    const double thr = frac * (k > 0 ? h->resid_total : 1.0);
     int sel = -1; double before = 0.0, run = 0.0;
     int last_pos_chunk = -1;
     for (int c0 = 0; c0 < nch && sel < 0; c0 += 32) {
@@ -54,7 +43,7 @@ __device__ int resample_draw(const Header* h, const ParamView& pv, int k, double
             const float2 ms = pv.chunk[c];
             R = (double)ms.y * exp((double)ms.x / T - lse);
             const int cb = chunk_begin(c, head), ce = chunk_end(c, head, nch, V);
-            for (int j = 0; j < k; j++) { const int id = pv.id[j]; if (id >= cb && id < ce) R -= pv.p[j]; }
+            for (int j = 0; j < k; j++) { const int id = s_id[j]; if (id >= cb && id < ce) R -= s_p[j]; }
             if (R < 0.0) R = 0.0;
         }
         const double inc = warp_incl_scan(R, lane) + run;
@@ -120,6 +109,8 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
 {
     __shared__ int s_lid[kVerifyWarps][kMaxSupport];
     __shared__ double s_lr[kVerifyWarps][kMaxSupport];
+    __shared__ int s_sid[kVerifyWarps][kMaxSupport];
+    __shared__ double s_sp[kVerifyWarps][kMaxSupport];
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int b = blockIdx.x * kVerifyWarps + wib;
     if (b >= batch) return;
@@ -141,7 +132,7 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
         if (k == 0) {
             // no rule was solved: emit a sample of the target distribution itself
             status = h->status;
-            token = resample_draw(h, pv, 0, u1, lane, s_lid[wib], s_lr[wib]);
+            token = resample_draw(h, pv, 0, u1, lane, s_lid[wib], s_lr[wib], s_sid[wib], s_sp[wib]);
             accepted = __any_sync(0xffffffffu, lane < n && tok == token) ? 1 : 0;
             if (token < 0) accepted = 0;
         } else {
@@ -188,7 +179,7 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
                     token = __shfl_sync(0xffffffffu, tok, 31 - __clz(posm));
                     accepted = 1;
                 } else {
-                    token = resample_draw(h, pv, k, u1, lane, s_lid[wib], s_lr[wib]);
+                    token = resample_draw(h, pv, k, u1, lane, s_lid[wib], s_lr[wib], s_sid[wib], s_sp[wib]);
                     accepted = 0;
                 }
             }
