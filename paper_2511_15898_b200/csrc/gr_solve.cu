@@ -33,7 +33,7 @@ constexpr double kStepClamp = 3.0;
 struct SolveLayout {
     int KP, n, Qt;
     // offsets in doubles
-    int d, tg, p, r, key, w, psi, Dr, alpha, alpha_prev, delta, g, g2, col, E, J, tq, cq, X, H, A, P, PP, gq, g2q, scal;
+    int d, tg, p, r, key, w, psi, Dr, alpha, alpha_prev, delta, g, g2, col, E, J, tq, cq, X, H, A, P, PP, PX, AX, gq, g2q, scal;
     int ints;      // offset in bytes of the int region
     int total_bytes;
     __host__ __device__ SolveLayout(int KP_, int n_, int Qt_) : KP(KP_), n(n_), Qt(Qt_) {
@@ -50,6 +50,8 @@ struct SolveLayout {
         A = o; o += Qt * (n + 1) * KP;
         P = o; o += Qt * (n + 1);
         PP = o; o += Qt * kGroups * (n + 1);
+        PX = o; o += Qt * 3 * (n + 1);
+        AX = o; o += Qt * (n + 1);
         gq = o; o += Qt * KP; g2q = o; o += Qt * KP;
         scal = o; o += 32;
         ints = o * 8;
@@ -66,7 +68,7 @@ __host__ int solve_smem_bytes(int KP, int n, int Qt) { return SolveLayout(KP, n,
 
 struct Sm {
     double *d, *tg, *p, *r, *key, *w, *psi, *Dr, *alpha, *alpha_prev, *delta, *g, *g2, *col, *E, *J, *tq, *cq, *X, *H,
-        *A, *P, *PP, *gq, *g2q, *scal;
+        *A, *P, *PP, *PX, *AX, *gq, *g2q, *scal;
     int *id, *blk, *order, *itmp;
     int KP, n, Qt;
 };
@@ -74,7 +76,7 @@ struct Sm {
 __device__ inline int tri(int i, int l) { return i * (i + 1) / 2 + l; }   // l <= i
 
 // scal[] slots
-enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SHI, S_S0, S_STEP, S_H };
+enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SHI, S_S0, S_STEP, S_H, S_DA, S_DB };
 
 // Evaluate g (and, if want_jac, the packed lower triangle of the Hessian) at sm.alpha[0..m).
 // d = draft masses of the system's tokens, hmass = draft mass of everything of higher ratio
@@ -99,6 +101,9 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
     double nfact = 1.0;
     for (int c = 2; c <= n; c++) nfact *= (double)c;
     const int gsz = (m + kGroups - 1) / kGroups;
+    // Dominant tokens (at most two; only for n > 16): the series division h = e / f would lose too many digits
+    // for them, so their leave-one-out products are multiplied out instead (all coefficients positive).
+    const int da = (int)sm.scal[S_DA], db = (int)sm.scal[S_DB];
 
     for (int q0 = 0; q0 < Q; q0 += Qt) {
         const int qn = min(Qt, Q - q0);
@@ -142,6 +147,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             double* PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
             const int j0 = grp * gsz, j1 = min(m, j0 + gsz);
             for (int j = j0; j < j1; j++) {
+                if (j == da || j == db) continue;          // dominant factors are applied after the tree
                 const double x = sm.X[q * KP + j];
                 for (int c = n; c >= 1; c--) {
                     double acc = 0.0;
@@ -166,11 +172,65 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             }
             __syncthreads();
         }
+        if (da >= 0) {
+            // PP[q][0] = product without the dominant factors (LAB).  PX[q][0] = all but a, PX[q][1] = all but b,
+            // PX[q][2] = full product.
+            for (int task = tid; task < qn * 3; task += kSolveThreads) {
+                const int q = task / 3, which = task - q * 3;
+                const double* Lab = sm.PP + (size_t)(q * kGroups) * n1;
+                double* out = sm.PX + (size_t)(q * 3 + which) * n1;
+                for (int c = 0; c <= n; c++) out[c] = Lab[c];
+                // factors to apply: which 0 -> f_b, which 1 -> f_a, which 2 -> f_a and f_b
+                for (int pass = 0; pass < 2; pass++) {
+                    const int j = pass == 0 ? ((which == 1 || which == 2) ? da : -1) : ((which == 0 || which == 2) ? db : -1);
+                    if (j < 0) continue;
+                    const double x = sm.X[q * KP + j];
+                    for (int c = n; c >= 1; c--) {
+                        double acc = 0.0;
+                        for (int a = 1; a <= c; a++) acc += sm.E[a * KP + j] * out[c - a];
+                        out[c] += x * acc;
+                    }
+                }
+            }
+            __syncthreads();
+        }
         // per (node, token): gradient integrand; series A = P h scaled for the Hessian
         for (int task = tid; task < qn * m; task += kSolveThreads) {
             const int q = task / m, j = task - q * m;
-            const double* Pq = sm.PP + (size_t)(q * kGroups) * n1;
+            const double* Pq = da >= 0 ? sm.PX + (size_t)(q * 3 + 2) * n1 : sm.PP + (size_t)(q * kGroups) * n1;
             double* Hq = sm.H + (size_t)q * n1 * KP;
+            if (j == da || j == db) {
+                // dominant token: dM/dx_j = n! [lambda^n] e_j L_j with L_j the product of all other factors
+                const double* Lj = sm.PX + (size_t)(q * 3 + (j == da ? 0 : 1)) * n1;
+                double val = 0.0;
+                for (int c = 1; c <= n; c++) val += Lj[n - c] * sm.E[c * KP + j];
+                const double u = sm.w[j] * sm.X[q * KP + j];
+                const double cg = sm.cq[q];
+                const double gi = cg * u * val;
+                sm.gq[q * KP + j] = gi;
+                sm.g2q[q * KP + j] = gi * sm.tq[q] * sm.w[j];
+                if (want_jac) {
+                    double* Aq = sm.A + (size_t)q * n1 * KP;
+                    const double sa = cg * sm.tq[q] * u;
+                    for (int e = 1; e < n; e++) {
+                        double acc = 0.0;
+                        for (int c = 1; c <= e; c++) acc += sm.E[c * KP + j] * Lj[e - c];
+                        Aq[e * KP + j] = sa * acc;
+                    }
+                    if (j == da && db >= 0) {
+                        // for the pair (a, b): the series e_a times the product without both
+                        const double* Lab = sm.PP + (size_t)(q * kGroups) * n1;
+                        double* Ax = sm.AX + (size_t)q * n1;
+                        for (int e = 1; e < n; e++) {
+                            double acc = 0.0;
+                            for (int c = 1; c <= e; c++) acc += sm.E[c * KP + j] * Lab[e - c];
+                            Ax[e] = sa * acc;
+                        }
+                    }
+                    for (int c = 1; c < n; c++) Hq[c * KP + j] = u * sm.E[c * KP + j];
+                }
+                continue;
+            }
             double val = 0.0;
             for (int c = 1; c <= n; c++) val += Pq[n - c] * Hq[c * KP + j];
             const double u = sm.w[j] * sm.X[q * KP + j];
@@ -200,10 +260,19 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             for (int i = 1 + warp; i < m; i += kSolveWarps) {
                 for (int l = lane; l < i; l += 32) {
                     double acc = 0.0;
+                    const bool domi = (i == da || i == db), doml = (l == da || l == db);
+                    // the A-series of a dominant token pairs with the h-series of the other token; two dominant
+                    // tokens pair through the product without both
+                    const int ia = (doml && !domi) ? l : i, ih = (doml && !domi) ? i : l;
                     for (int q = 0; q < qn; q++) {
                         const double* Aq = sm.A + (size_t)q * n1 * KP;
                         const double* Hq = sm.H + (size_t)q * n1 * KP;
-                        for (int c = 1; c < n; c++) acc += Aq[(n - c) * KP + i] * Hq[c * KP + l];
+                        if (domi && doml) {
+                            const double* Ax = sm.AX + (size_t)q * n1;
+                            for (int c = 1; c < n; c++) acc += Ax[n - c] * Hq[c * KP + db];
+                        } else {
+                            for (int c = 1; c < n; c++) acc += Aq[(n - c) * KP + ia] * Hq[c * KP + ih];
+                        }
                     }
                     sm.J[tri(i, l)] -= acc;
                 }
@@ -273,6 +342,21 @@ __device__ int solve_system(const Sm& sm, int m, const double* d, const double* 
         double pw = 1.0, fc = 1.0;
         sm.E[tid] = 0.0;
         for (int c = 1; c <= n; c++) { pw *= d[tid]; fc *= (double)c; sm.E[c * KP + tid] = pw / fc; }
+    }
+    // dominant tokens: d_j / (total mass) >= pi (1e5 / n!)^(1/n), checked only for n > 16 (below, the series
+    // division is accurate to 1e-11 for any token)
+    if (tid == 0) {
+        int a = -1, b2 = -1;
+        if (n > 16) {
+            double T = hmass, lf = 0.0;
+            for (int j = 0; j < m; j++) T += d[j];
+            for (int c = 2; c <= n; c++) lf += log((double)c);
+            const double thr = 3.141592653589793 * exp((log(1.0e5) - lf) / (double)n);
+            for (int j = 0; j < m; j++) {
+                if (d[j] >= thr * T) { if (a < 0) a = j; else if (b2 < 0) b2 = j; }
+            }
+        }
+        sm.scal[S_DA] = (double)a; sm.scal[S_DB] = (double)b2;
     }
     // starting point: the single-token balance  w/(1+w) * Pr[i in set(omega)] = rhs
     double a0 = 0.0;
@@ -385,6 +469,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     sm.alpha_prev = base + L.alpha_prev; sm.delta = base + L.delta; sm.g = base + L.g; sm.g2 = base + L.g2;
     sm.col = base + L.col; sm.E = base + L.E; sm.J = base + L.J; sm.tq = base + L.tq; sm.cq = base + L.cq;
     sm.X = base + L.X; sm.H = base + L.H; sm.A = base + L.A; sm.P = base + L.P; sm.PP = base + L.PP;
+    sm.PX = base + L.PX; sm.AX = base + L.AX;
     sm.gq = base + L.gq; sm.g2q = base + L.g2q; sm.scal = base + L.scal;
     int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
     sm.id = ib; sm.blk = ib + KP; sm.order = ib + 2 * KP; sm.itmp = ib + 3 * KP;

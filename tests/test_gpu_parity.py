@@ -189,3 +189,16 @@ def test_config4_whole_vocabulary_cells_alpha_star(n, sigma):
         a, _ = O.alpha_star_only(tl[b], dl[b], wl.n, wl.topk, wl.temp_target, wl.temp_draft)
         assert abs(float(solved.alpha_star[b]) - a) <= ALPHA_TOL, (b, float(solved.alpha_star[b]), a)
     assert bool((ver.token >= 0).all())
+
+
+def test_n32_with_a_dominant_draft_token_converges():
+    """n = 32: tokens holding a large share of the draft mass need the multiplied-out leave-one-out products
+    (the series division loses too many digits there); every instance must converge, and match the oracle."""
+    wl = W.config4(32, 20, 1.0, batch=96, device="cuda")
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+    torch.cuda.synchronize()
+    assert solved.status.cpu().tolist() == [G.GR_OK] * 96
+    top = torch.softmax(torch.topk(wl.p_logits, 20, dim=1).values.double(), dim=1)[:, 0]
+    assert float(top.max()) > 0.5          # the workload does contain dominant tokens
+    idx = torch.argsort(top, descending=True)[:6].tolist()
+    _check(P.compare(wl.rows(idx)))
