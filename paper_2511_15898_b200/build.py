@@ -9,8 +9,11 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgr_b200.so")
-SOURCES = ["gr_api.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_fullsort.cu", "gr_verify.cu"]
-HEADERS = [os.path.join(CSRC, "gr_common.cuh"), os.path.join(CSRC, "gr_prep.cuh"), os.path.join(ROOT, "include", "gr.h")]
+OBJ = os.path.join(HERE, "_build")
+SOURCES = ["gr_api.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_fast_n4.cu", "gr_fast_n8.cu",
+           "gr_fast_n16.cu", "gr_fullsort.cu", "gr_verify.cu"]
+HEADERS = [os.path.join(CSRC, "gr_common.cuh"), os.path.join(CSRC, "gr_prep.cuh"), os.path.join(CSRC, "gr_fast.cuh"),
+           os.path.join(ROOT, "include", "gr.h")]
 
 
 def _nvcc() -> str:
@@ -29,19 +32,40 @@ def needs_build() -> bool:
 
 
 def build_library(force: bool = False, verbose: bool = False) -> str:
+    """Compile each source to an object (in parallel; objects newer than every source and header are kept),
+    then link the shared library."""
     if not force and not needs_build():
         return LIB
-    cmd = [_nvcc(), "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
-           "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    os.makedirs(OBJ, exist_ok=True)
+    flags = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
+             "-I", os.path.join(ROOT, "include"), "-I", CSRC]
     if verbose:
-        cmd += ["-Xptxas", "-v"]
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose:
-        sys.stderr.write(res.stderr)
+        flags += ["-Xptxas", "-v"]
+    hdr_time = max(os.path.getmtime(h) for h in HEADERS)
+    jobs = []
+    objs = []
+    for s in SOURCES:
+        src = os.path.join(CSRC, s)
+        obj = os.path.join(OBJ, s[:-3] + ".o")
+        objs.append(obj)
+        fresh = (not force and not verbose and os.path.exists(obj)
+                 and os.path.getmtime(obj) > max(os.path.getmtime(src), hdr_time))
+        if not fresh:
+            jobs.append((s, subprocess.Popen([_nvcc()] + flags + ["-c", src, "-o", obj], stdout=subprocess.PIPE,
+                                             stderr=subprocess.STDOUT, text=True)))
+    failed = []
+    for s, proc in jobs:
+        out, _ = proc.communicate()
+        if verbose:
+            sys.stderr.write(out)
+        if proc.returncode != 0:
+            failed.append(s + ":\n" + out)
+    if failed:
+        raise RuntimeError("nvcc failed:\n" + "\n".join(failed))
+    res = subprocess.run([_nvcc(), "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a"]
+                         + objs + ["-o", LIB], capture_output=True, text=True)
     if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+        raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     return LIB
 
 

@@ -1,0 +1,808 @@
+// Fast per-instance solve for supports up to 64 tokens and n <= 16 (one 128-thread CTA per
+// instance, several CTAs per SM).
+//
+// Same mathematics as the robust kernel (gr_solve.cu): the gradient of the convex functions
+// of the inner system / of an outer block (Thm "Inner Convex Solver", Thm "Outer Convex Solver")
+// is the one-dimensional integral
+//   g_i = w_i int e^{-t slack} x_i(t) n! [lambda^n] P(lambda; t) h_i(lambda; t) dt,
+// and Newton's method on alpha = log w uses its exact Hessian.  Organised for throughput:
+//   - one warp per quadrature node, one lane per token (two tokens per lane above 32): every
+//     power series lives in registers;
+//   - the product P = e^{lambda h} prod_j f_j over the tokens is not multiplied out:
+//     d/dlambda log f_j = x_j d_j (1 + (1 - x_j) h_j), so the log-derivative S of P is a SUM over
+//     tokens (a warp reduction) and P follows from P' = S P.  In fp64 this is accurate to
+//     ~1e-12 for n <= 16 and degrades beyond (larger n takes the robust kernel);
+//   - h_j(lambda) = H(d_j lambda; x_j) with H(mu; x) = (e^mu - 1) / (1 + x (e^mu - 1)), whose
+//     coefficients obey a recurrence with compile-time constants 1/c!;
+//   - the Hessian's off-diagonal part  - sum_q c_q t_q (w x)_i (w x)_l n! [lambda^n] P h_i h_l  is a
+//     dense contraction over (node, series index); it only steers the iteration, so it is
+//     taken on every second node (trapezoid step doubled) and accumulated in fp32 from operands
+//     staged in shared memory; the gradient itself stays fp64 on every node;
+//   - the iteration starts from a mean-field point (each token against the expected weight
+//     of the other drafted tokens).
+#pragma once
+#include "gr_prep.cuh"
+
+namespace gr {
+
+constexpr int kFT = 128;              // threads per CTA
+constexpr int kFW = kFT / 32;         // warps per CTA
+constexpr int kMP = 64;               // padded support size of this kernel
+constexpr int kJC = 8;                // Hessian nodes staged per chunk
+constexpr double kFTEnd = 25.0;       // quadrature range constants, identical to the robust kernel's
+constexpr double kFDrop = 1.0;
+constexpr double kFTail = 3.0;
+constexpr int kFMaxNodes = 128;
+constexpr int kMS = 72;               // row stride of the staged operands (floats): conflict-free MMA fragment loads
+constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
+constexpr double kFAlphaClamp = 80.0;
+constexpr double kFStepClamp = 3.0;
+constexpr int kFSweeps = 3;           // fixed-point sweeps of the mean-field start
+
+struct FastLayout {
+    int KP;
+    int d, tg, p, r, key, psi, Dr, alpha, alpha_prev, delta, w, g, g2, col, gw, g2w, tq, cq, scal, uni;
+    int jacc_bytes_off, ints, total_bytes;
+    __host__ __device__ FastLayout(int KP_, int NT) : KP(KP_) {
+        int o = 0;
+        d = o; o += KP; tg = o; o += KP; p = o; o += KP; r = o; o += KP; key = o; o += KP;
+        psi = o; o += KP + 4; Dr = o; o += KP + 4;
+        alpha = o; o += KP; alpha_prev = o; o += KP; delta = o; o += KP; w = o; o += KP; g = o; o += KP;
+        g2 = o; o += KP; col = o; o += kMP;
+        gw = o; o += kFW * KP; g2w = o; o += kFW * KP;
+        tq = o; o += kFMaxNodes; cq = o; o += kFMaxNodes;
+        scal = o; o += 32;
+        uni = o;
+        // union: staging of the Hessian operands (two float arrays [kJC * NT][kMS]) / vectors of the Newton step
+        const int stage_doubles = (2 * kJC * NT * kMS * 4 + 7) / 8;
+        const int jmat_doubles = 2 * (kMP + 4) + 2 * kMP;    // (floats, so twice what is needed) pivot row / column buffers
+        o += stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
+        jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
+        o += (kMP * (kMP + 1) + 1) / 2;
+        ints = o * 8;
+        total_bytes = ints + KP * 3 * 4 + 64;
+    }
+};
+static inline int fast_smem_bytes(int KP, int NT) { return FastLayout(KP, NT).total_bytes; }
+
+struct FSm {
+    double *d, *tg, *p, *r, *key, *psi, *Dr, *alpha, *alpha_prev, *delta, *w, *g, *g2, *col, *gw, *g2w, *tq, *cq,
+        *scal, *J;
+    float *AS, *HS, *Jacc;
+    int *id, *blk, *itmp;
+    int KP;
+};
+enum { SC_Q = 0, SC_FAIL = 1, SC_RED = 8 };
+
+__device__ __forceinline__ double ipow(double x, int n) {
+    double r = 1.0;
+    while (n > 0) { if (n & 1) r *= x; x *= x; n >>= 1; }
+    return r;
+}
+
+// exp(-y) for y >= 0 (fp64): range reduction by ln 2 and a degree-13 Taylor polynomial on |r| <= ln2/2
+// (truncation below 1e-17 relative); results below 2^-1000 are flushed to zero.
+__device__ __forceinline__ double exp_neg(double y)
+{
+    const double t = -y;
+    const double kf = rint(t * 1.4426950408889634);
+    if (kf < -1000.0) return 0.0;
+    double r = fma(-kf, 6.93147180369123816490e-01, t);
+    r = fma(-kf, 1.90821492927058770002e-10, r);
+    double p = 1.6059043836821613e-10;                 // 1/13!
+    p = fma(p, r, 2.08767569878681e-09);               // 1/12!
+    p = fma(p, r, 2.505210838544172e-08);              // 1/11!
+    p = fma(p, r, 2.755731922398589e-07);              // 1/10!
+    p = fma(p, r, 2.7557319223985893e-06);             // 1/9!
+    p = fma(p, r, 2.48015873015873e-05);               // 1/8!
+    p = fma(p, r, 1.984126984126984e-04);              // 1/7!
+    p = fma(p, r, 1.388888888888889e-03);              // 1/6!
+    p = fma(p, r, 8.333333333333333e-03);              // 1/5!
+    p = fma(p, r, 4.1666666666666664e-02);             // 1/4!
+    p = fma(p, r, 1.6666666666666666e-01);             // 1/3!
+    p = fma(p, r, 0.5);
+    p = fma(p, r, 1.0);
+    p = fma(p, r, 1.0);
+    const int k = (int)kf;
+    return __hiloint2double(__double2hiint(p) + (k << 20), __double2loint(p));
+}
+
+__device__ __forceinline__ constexpr double inv_fact(int c) {
+    double f = 1.0;
+    for (int i = 2; i <= c; i++) f *= (double)i;
+    return 1.0 / f;
+}
+
+// hh[c], c = 1..NT: coefficients of (e^mu - 1) / (1 + x (e^mu - 1)) in mu.  Column-oriented so that the
+// dependent chain is two operations per coefficient.
+template <int NT>
+__device__ __forceinline__ void unit_h_series(double x, double* hh)
+{
+    double acc[NT + 1];
+#pragma unroll
+    for (int c = 1; c <= NT; c++) acc[c] = 0.0;
+    hh[1] = 1.0;
+#pragma unroll
+    for (int k = 1; k < NT; k++) {
+#pragma unroll
+        for (int c = k + 1; c <= NT; c++) acc[c] = fma(inv_fact(c - k), hh[k], acc[c]);
+        hh[k + 1] = fma(-x, acc[k + 1], inv_fact(k + 1));
+    }
+}
+
+__device__ __forceinline__ double warp_sum_d(double v) {
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Sum of NT-entry vectors over the 32 lanes, result in every lane.  Recursive halving: at each of the
+// first log2(NT) levels a lane keeps half of its entries and hands the other half to its partner, so the
+// exchange costs NT - 1 + (5 - log2 NT) shuffles instead of 5 NT; an all-gather of NT shuffles follows.
+template <int NT>
+__device__ __forceinline__ void warp_allreduce_series(double* S, int lane)
+{
+    static_assert(NT == 4 || NT == 8 || NT == 16, "series length");
+    int cnt = NT, o = 16;
+#pragma unroll
+    for (int lvl = 0; lvl < (NT == 16 ? 4 : (NT == 8 ? 3 : 2)); lvl++) {
+        const int half = cnt >> 1;
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int c = 0; c < NT / 2; c++) {
+            if (c < half) {
+                const double keep = up ? S[c + half] : S[c];
+                const double send = up ? S[c] : S[c + half];
+                S[c] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+            }
+        }
+        cnt = half; o >>= 1;
+    }
+    double v = S[0];
+    for (; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    // lane bits (4, 3[, 2[, 1]]) say which entry the lane holds
+#pragma unroll
+    for (int c = 0; c < NT; c++) {
+        const int src = (NT == 16) ? ((((c >> 3) & 1) << 4) | (((c >> 2) & 1) << 3) | (((c >> 1) & 1) << 2) | ((c & 1) << 1))
+                      : (NT == 8) ? ((((c >> 2) & 1) << 4) | (((c >> 1) & 1) << 3) | ((c & 1) << 2))
+                                  : ((((c >> 1) & 1) << 4) | ((c & 1) << 3));
+        S[c] = __shfl_sync(0xffffffffu, v, src);
+    }
+}
+
+// tf32 rounding of a staged operand (the contraction runs on the tensor cores: it is the one dense
+// contraction of the path, and it only steers Newton's method)
+__device__ __forceinline__ float to_tf32(float x) {
+    uint32_t u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(x));
+    return __uint_as_float(u);
+}
+
+// Series of length 16 cancel too strongly for one tf32 product (a dominant draft token makes the terms of
+// sum_kappa A[n - kappa] h[kappa] alternate at ~1e3 times their sum): their operands are staged in full fp32 and
+// split into two tf32 parts when the fragments are loaded (three MMAs per tile step, error ~1e-6 per term).
+template <int NT>
+__device__ __forceinline__ float stage_round(float x) { return NT > 8 ? x : to_tf32(x); }
+
+__device__ __forceinline__ void mma_tf32(float& c0, float& c1, float& c2, float& c3, uint32_t a0, uint32_t a1,
+                                         uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c0), "+f"(c1), "+f"(c2), "+f"(c3)
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// One chunk of the Hessian contraction: Jacc[i][l] += sum over the staged rows kk of AS[kk][i] HS[kk][l] for the
+// 16 x 8 tiles that touch the lower triangle, as m16n8k8 tf32 MMAs with fp32 accumulation.  K8 = staged rows,
+// a multiple of 8.  The 20 lower tiles of the 64 x 64 matrix are dealt round-robin to the four warps.
+template <bool kSplit>
+__device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gid = lane >> 2, tig = lane & 3;
+    for (int t = warp; t < 20; t += kFW) {
+        const int mi = t >= 12 ? 3 : (t >= 6 ? 2 : (t >= 2 ? 1 : 0));
+        const int ni = t - (mi == 3 ? 12 : (mi == 2 ? 6 : (mi == 1 ? 2 : 0)));
+        const int i0 = 16 * mi, l0 = 8 * ni;
+        if (i0 >= m || l0 >= m) continue;
+        float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
+        for (int k0 = 0; k0 < K8; k0 += 8) {
+            const float* Ap = sm.AS + (k0 + tig) * kMS + i0 + gid;
+            const float* Bp = sm.HS + (k0 + tig) * kMS + l0 + gid;
+            const float fa[4] = {Ap[0], Ap[8], Ap[4 * kMS], Ap[4 * kMS + 8]};
+            const float fb[2] = {Bp[0], Bp[4 * kMS]};
+            if (kSplit) {
+                uint32_t ah[4], al[4], bh[2], bl[2];
+#pragma unroll
+                for (int z = 0; z < 4; z++) {
+                    const float hi = to_tf32(fa[z]);
+                    ah[z] = __float_as_uint(hi); al[z] = __float_as_uint(to_tf32(fa[z] - hi));
+                }
+#pragma unroll
+                for (int z = 0; z < 2; z++) {
+                    const float hi = to_tf32(fb[z]);
+                    bh[z] = __float_as_uint(hi); bl[z] = __float_as_uint(to_tf32(fb[z] - hi));
+                }
+                mma_tf32(c0, c1, c2, c3, al[0], al[1], al[2], al[3], bh[0], bh[1]);
+                mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bl[0], bl[1]);
+                mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bh[0], bh[1]);
+            } else {
+                mma_tf32(c0, c1, c2, c3, __float_as_uint(fa[0]), __float_as_uint(fa[1]), __float_as_uint(fa[2]),
+                         __float_as_uint(fa[3]), __float_as_uint(fb[0]), __float_as_uint(fb[1]));
+            }
+        }
+        float* J0 = sm.Jacc + (i0 + gid) * kJS + l0 + 2 * tig;
+        J0[0] += c0; J0[1] += c1;
+        J0[8 * kJS] += c2; J0[8 * kJS + 1] += c3;
+    }
+}
+
+// g (always), and with want_jac the diagonal part g2 and the contraction Jacc, at the weights in sm.w.
+// The contraction takes every jstride-th node (weights scaled by jstride).
+// Node abscissae / weights are in sm.tq / sm.cq, their number in sm.scal[SC_Q].
+template <int NT, int TPL>
+__device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double hmass, bool want_jac, int jstride)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, KP = sm.KP;
+    const int Q = (int)sm.scal[SC_Q];
+    double wr[TPL], dr[TPL], gacc[TPL], g2acc[TPL];
+#pragma unroll
+    for (int tt = 0; tt < TPL; tt++) {
+        const int j = lane + 32 * tt;
+        wr[tt] = j < m ? sm.w[j] : 0.0;
+        dr[tt] = j < m ? d[j] : 0.0;
+        gacc[tt] = 0.0; g2acc[tt] = 0.0;
+    }
+    if (want_jac) {
+        for (int e = tid; e < kMP * kJS; e += kFT) sm.Jacc[e] = 0.f;
+    }
+    const int span = jstride * kJC;      // nodes per chunk: every jstride-th one is a Hessian node
+    for (int q0 = 0; q0 < Q; q0 += span) {
+        const int q1 = min(Q, q0 + span);
+        for (int q = q0 + warp; q < q1; q += kFW) {
+            const double t = sm.tq[q];
+            double S[NT];
+#pragma unroll
+            for (int c = 0; c < NT; c++) S[c] = 0.0;
+            double xk[TPL];
+#pragma unroll
+            for (int tt = 0; tt < TPL; tt++) {
+                const double x = exp_neg(t * wr[tt]);
+                xk[tt] = x;
+                double hh[NT + 1];
+                unit_h_series<NT>(x, hh);
+                // h[c] = d^c hh[c];  S[0] += x d,  S[c] += x (1 - x) d h[c]
+                const double dd = dr[tt];
+                S[0] = fma(x, dd, S[0]);
+                double pw = x * (1.0 - x) * dd;
+#pragma unroll
+                for (int c = 1; c < NT; c++) {
+                    pw *= dd;
+                    S[c] = fma(pw, hh[c], S[c]);
+                }
+            }
+            // log-derivative of the product: sum over the tokens (all lanes end with the totals)
+            warp_allreduce_series<NT>(S, lane);
+            S[0] += hmass;
+            // P' = S P, column-oriented
+            double P[NT + 1], acc[NT + 1];
+            P[0] = 1.0;
+#pragma unroll
+            for (int c = 1; c <= NT; c++) acc[c] = 0.0;
+#pragma unroll
+            for (int k = 0; k < NT; k++) {
+#pragma unroll
+                for (int c = k + 1; c <= NT; c++) acc[c] = fma(S[c - 1 - k], P[k], acc[c]);
+                P[k + 1] = acc[k + 1] * (1.0 / (double)(k + 1));
+            }
+            // R[c] = P[n - c]: the coefficient that pairs with h[c] in [lambda^n] P h
+            // (for n < NT: the reversed series moved down by NT - n places, one conditional move per bit)
+            double R[NT + 1];
+#pragma unroll
+            for (int c = 1; c <= NT; c++) R[c] = P[NT - c];
+            if (n != NT) {
+                const int sh = NT - n;
+#pragma unroll
+                for (int bit = NT / 2; bit >= 1; bit >>= 1) {
+                    if (sh & bit) {
+#pragma unroll
+                        for (int c = 1; c <= NT; c++) R[c] = (c + bit <= NT) ? R[c + bit] : 0.0;
+                    }
+                }
+            }
+            const double cq = sm.cq[q];
+            const bool jnode = want_jac && ((q - q0) % jstride == 0);
+            const int slot = (q - q0) / jstride;
+#pragma unroll
+            for (int tt = 0; tt < TPL; tt++) {
+                double hh[NT + 1], hd[NT + 1];
+                unit_h_series<NT>(xk[tt], hh);
+                const double dd = dr[tt];
+                double pw = 1.0, val = 0.0;
+#pragma unroll
+                for (int c = 1; c <= NT; c++) {
+                    pw *= dd;
+                    hd[c] = pw * hh[c];                 // h[c] = d^c hh[c]
+                    val = fma(R[c], hd[c], val);
+                }
+                const double u = wr[tt] * xk[tt];
+                const double gi = cq * u * val;
+                gacc[tt] += gi;
+                g2acc[tt] = fma(gi * t, wr[tt], g2acc[tt]);
+                if (jnode) {
+                    // A = P h (series), paired as  sum_kappa A[n - kappa] h_l[kappa],  kappa = 1..n-1.
+                    // Staged scaled: AS = 2 c_q t u A[n - kappa] (the 2: every second node), HS = u h[kappa].
+                    // Row kappa - 1 of the node's slot holds the pair (A[n - kappa], h[kappa]); rows n - 1 .. NT - 1
+                    // are zero (they pad the contraction length to a multiple of the MMA depth).
+                    const int j = lane + 32 * tt;
+                    const double sa = (double)jstride * cq * t * u;
+                    float* as = sm.AS + slot * NT * kMS + j;
+                    float* hs = sm.HS + slot * NT * kMS + j;
+                    if (n == NT) {
+                        // full series length: fixed rows, each A consumed as soon as it is formed
+#pragma unroll
+                        for (int kap = 1; kap < NT; kap++) {
+                            double a = 0.0;              // A[NT - kap] = sum_c h[c] P[NT - kap - c]
+#pragma unroll
+                            for (int c = 1; c <= NT - kap; c++) a = fma(hd[c], P[NT - kap - c], a);
+                            as[(kap - 1) * kMS] = stage_round<NT>((float)(sa * a));
+                            hs[(kap - 1) * kMS] = stage_round<NT>((float)(u * hd[kap]));
+                            if (TPL == 1) { as[(kap - 1) * kMS + 32] = 0.f; hs[(kap - 1) * kMS + 32] = 0.f; }
+                        }
+                        as[(NT - 1) * kMS] = 0.f; hs[(NT - 1) * kMS] = 0.f;
+                        if (TPL == 1) { as[(NT - 1) * kMS + 32] = 0.f; hs[(NT - 1) * kMS + 32] = 0.f; }
+                    } else {
+#pragma unroll
+                        for (int e2 = 1; e2 < NT; e2++) {
+                            double a = 0.0;              // A[e2] = sum_{c=1..e2} h[c] P[e2 - c]
+#pragma unroll
+                            for (int c = 1; c <= e2; c++) a = fma(hd[c], P[e2 - c], a);
+                            if (e2 < n) as[(n - e2 - 1) * kMS] = stage_round<NT>((float)(sa * a));
+                        }
+#pragma unroll
+                        for (int kap = 1; kap <= NT; kap++) {
+                            const bool live = kap < n;
+                            if (!live) as[(kap - 1) * kMS] = 0.f;
+                            hs[(kap - 1) * kMS] = live ? stage_round<NT>((float)(u * hd[kap])) : 0.f;
+                            if (TPL == 1) { as[(kap - 1) * kMS + 32] = 0.f; hs[(kap - 1) * kMS + 32] = 0.f; }
+                        }
+                    }
+                }
+            }
+        }
+        if (want_jac) {
+            const int nstaged = (q1 - q0 + jstride - 1) / jstride;
+            int K8 = nstaged * NT;
+            if (K8 & 7) {
+                // NT = 4 with an odd number of staged nodes: one more all-zero slot completes the MMA depth
+                for (int e = tid; e < NT * kMS; e += kFT) { sm.AS[K8 * kMS + e] = 0.f; sm.HS[K8 * kMS + e] = 0.f; }
+                K8 += NT;
+            }
+            __syncthreads();
+            hess_chunk<(NT > 8)>(sm, K8, m);
+            __syncthreads();
+        }
+    }
+#pragma unroll
+    for (int tt = 0; tt < TPL; tt++) {
+        const int j = lane + 32 * tt;
+        if (j < m) { sm.gw[warp * KP + j] = gacc[tt]; sm.g2w[warp * KP + j] = g2acc[tt]; }
+    }
+    __syncthreads();
+    if (tid < m) {
+        double a = 0.0, b2 = 0.0;
+#pragma unroll
+        for (int w2 = 0; w2 < kFW; w2++) { a += sm.gw[w2 * KP + tid]; b2 += sm.g2w[w2 * KP + tid]; }
+        sm.g[tid] = a; sm.g2[tid] = b2;
+    }
+    __syncthreads();
+}
+
+// w = exp(alpha), its range, and the quadrature grid for it.
+static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
+{
+    const int tid = threadIdx.x;
+    double* red = sm.scal + SC_RED;
+    double a = 0.0;
+    if (tid < m) { a = sm.alpha[tid]; sm.w[tid] = exp(a); }
+    // extreme alphas in one pass (they give the extreme weights)
+    double hi = tid < m ? a : -1.0e300, lo = tid < m ? -a : -1.0e300;
+    for (int o = 16; o > 0; o >>= 1) {
+        hi = fmax(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        lo = fmax(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    }
+    __syncthreads();
+    if ((tid & 31) == 0) { red[2 * (tid >> 5)] = hi; red[2 * (tid >> 5) + 1] = lo; }
+    __syncthreads();
+    hi = red[0]; lo = red[1];
+#pragma unroll
+    for (int i = 1; i < kFW; i++) { hi = fmax(hi, red[2 * i]); lo = fmax(lo, red[2 * i + 1]); }
+    lo = -lo;
+    const double wmax = exp(hi), wmin = exp(lo);
+    const double rate = slack ? 1.0 + wmin : wmin;
+    const double s_hi = log(kFTEnd / rate);
+    const double s0 = -log((slack ? 1.0 : 0.0) + wmax) - kFDrop;
+    int Q = (int)ceil((s_hi - (s0 - kFTail)) / qstep) + 1;
+    if (Q > kFMaxNodes) Q = kFMaxNodes;
+    double nfact = 1.0;
+    for (int c = 2; c <= n; c++) nfact *= (double)c;
+    for (int q = tid; q < Q; q += kFT) {
+        const double s = s_hi - qstep * (double)q;
+        const double e = exp(-(s - s0));
+        const double t = exp(s - e);
+        sm.tq[q] = t;
+        sm.cq[q] = qstep * (1.0 + e) * t * (slack ? exp(-t) : 1.0) * nfact;
+    }
+    if (tid == 0) sm.scal[SC_Q] = (double)Q;
+    __syncthreads();
+}
+
+// Newton step: fp32 Cholesky of the Hessian in place in the contraction accumulator (row stride kJS),
+// with the forward substitution carried along and the backward substitution on warp 0.  The step only
+// steers the iteration (the fp64 gradient decides convergence) and the Hessian was accumulated in fp32.
+// Thread (ty, tx) = (tid / 8, tid % 8) updates the trailing rows j+1+ty+16a and columns j+1+tx+8b.
+// Matrix: off-diagonal -Jacc (lower triangle), diagonal g - g2, plus `add` everywhere.  Writes the step
+// into sm.delta; sets SC_FAIL when a pivot is not positive.
+static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
+{
+    const int tid = threadIdx.x, ty = tid >> 3, tx = tid & 7;
+    float* Jm = sm.Jacc;
+    float* yv = reinterpret_cast<float*>(sm.J);        // [kMP] working right-hand side
+    float* yf = yv + kMP;                              // [kMP] forward-substituted right-hand side, then the solution
+    float* dg = yf + kMP;                              // [kMP] diagonal of the factor
+    const float addf = (float)add;
+    for (int e = tid; e < m * kMP; e += kFT) {
+        const int i = e >> 6, l = e & (kMP - 1);
+        if (l < i) Jm[i * kJS + l] = addf - Jm[i * kJS + l];
+    }
+    if (tid < m) {
+        Jm[tid * kJS + tid] = (float)(sm.g[tid] - sm.g2[tid]) + addf;
+        yv[tid] = -(float)(sm.g[tid] - rhs[tid]);
+    }
+    __syncthreads();
+    bool bad = false;
+    // blocked right-looking factorisation, four columns per pair of barriers
+    for (int j0 = 0; j0 < m; j0 += 4) {
+        const int nb = min(4, m - j0);
+        // every thread factors the diagonal block (at most 4 x 4) in registers
+        float Lb[4][4], yb[4], dinv[4];
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+#pragma unroll
+            for (int c2 = 0; c2 <= c; c2++) Lb[c][c2] = (c < nb) ? Jm[(j0 + c) * kJS + j0 + c2] : (c == c2 ? 1.f : 0.f);
+            yb[c] = (c < nb) ? yv[j0 + c] : 0.f;
+        }
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+            float dv = Lb[c][c];
+#pragma unroll
+            for (int e2 = 0; e2 < c; e2++) dv = fmaf(-Lb[c][e2], Lb[c][e2], dv);
+            if (!(dv > 0.f)) bad = true;
+            dinv[c] = rsqrtf(dv);
+            Lb[c][c] = dv * dinv[c];
+            float yc = yb[c];
+#pragma unroll
+            for (int e2 = 0; e2 < c; e2++) yc = fmaf(-Lb[c][e2], yb[e2], yc);
+            yb[c] = yc * dinv[c];
+#pragma unroll
+            for (int r2 = c + 1; r2 < 4; r2++) {
+                float v = Lb[r2][c];
+#pragma unroll
+                for (int e2 = 0; e2 < c; e2++) v = fmaf(-Lb[r2][e2], Lb[c][e2], v);
+                Lb[r2][c] = v * dinv[c];
+            }
+        }
+        if (bad) break;
+        __syncthreads();                       // every thread has read the block before it is overwritten
+        // panel below the block: one row per thread
+        const int i1 = j0 + nb + tid;
+        if (i1 < m) {
+            float lp[4];
+            float yi = yv[i1];
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                float v = (c < nb) ? Jm[i1 * kJS + j0 + c] : 0.f;
+#pragma unroll
+                for (int e2 = 0; e2 < c; e2++) v = fmaf(-lp[e2], Lb[c][e2], v);
+                lp[c] = v * dinv[c];
+                if (c < nb) { Jm[i1 * kJS + j0 + c] = lp[c]; yi = fmaf(-lp[c], yb[c], yi); }
+            }
+            yv[i1] = yi;
+        }
+        if (tid == kFT - 1) {
+#pragma unroll
+            for (int c = 0; c < 4; c++) {
+                if (c < nb) {
+                    dg[j0 + c] = Lb[c][c]; yf[j0 + c] = yb[c];
+#pragma unroll
+                    for (int c2 = 0; c2 < c; c2++) Jm[(j0 + c) * kJS + j0 + c2] = Lb[c][c2];
+                }
+            }
+        }
+        __syncthreads();
+        // trailing update  J[i][l] -= sum_c L[i][c] L[l][c],  j0 + nb <= l <= i
+        const int t0 = j0 + nb;
+        float cl[8][4];
+#pragma unroll
+        for (int b2 = 0; b2 < 8; b2++) {
+            const int l = t0 + tx + 8 * b2;
+#pragma unroll
+            for (int c = 0; c < 4; c++) cl[b2][c] = (l < m && c < nb) ? Jm[l * kJS + j0 + c] : 0.f;
+        }
+        for (int i = t0 + ty; i < m; i += 16) {
+            float* row = Jm + i * kJS;
+            float ci[4];
+#pragma unroll
+            for (int c = 0; c < 4; c++) ci[c] = (c < nb) ? row[j0 + c] : 0.f;
+#pragma unroll
+            for (int b2 = 0; b2 < 8; b2++) {
+                const int l = t0 + tx + 8 * b2;
+                if (l <= i) {
+                    float v = row[l];
+#pragma unroll
+                    for (int c = 0; c < 4; c++) v = fmaf(-ci[c], cl[b2][c], v);
+                    row[l] = v;
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (bad) {
+        if (tid == 0) sm.scal[SC_FAIL] = 1.0;
+        __syncthreads();
+        return;
+    }
+    // backward substitution L^T x = y on warp 0, four unknowns at a time: every lane solves the 4 x 4
+    // triangle redundantly, then the lanes update the unknowns above it
+    if (tid < 32) {
+        for (int e0 = ((m - 1) >> 2) << 2; e0 >= 0; e0 -= 4) {
+            const int nb = min(4, m - e0);
+            float x[4];
+#pragma unroll
+            for (int c = 3; c >= 0; c--) {
+                float v = 0.f;
+                if (c < nb) {
+                    v = yf[e0 + c];
+#pragma unroll
+                    for (int c2 = 3; c2 > c; c2--)
+                        if (c2 < nb) v = fmaf(-Jm[(e0 + c2) * kJS + e0 + c], x[c2], v);
+                    v = v / dg[e0 + c];
+                }
+                x[c] = v;
+            }
+            __syncwarp();
+            if (tid < nb) yf[e0 + tid] = tid == 0 ? x[0] : (tid == 1 ? x[1] : (tid == 2 ? x[2] : x[3]));
+            for (int l = tid; l < e0; l += 32) {
+                float v = yf[l];
+#pragma unroll
+                for (int c = 0; c < 4; c++)
+                    if (c < nb) v = fmaf(-Jm[(e0 + c) * kJS + l], x[c], v);
+                yf[l] = v;
+            }
+            __syncwarp();
+        }
+    }
+    __syncthreads();
+    if (tid < m) sm.delta[tid] = (double)yf[tid];
+    __syncthreads();
+}
+
+// Newton iteration for one system.  On return sm.w holds exp(alpha) at the last evaluated point.
+template <int NT, int TPL>
+__device__ int fast_system(const FSm& sm, int m, int n, const double* d, const double* rhs, double hmass, int slack,
+                           double tol, int max_iters, double qstep, double* gnorm, int* iters)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double* red = sm.scal + SC_RED;
+    // ---- mean-field starting point: token i wins the share w_i / (slack + w_i + S_i) of the tuples that
+    //      contain it, S_i = expected weight of the other drafted tokens given that i was drafted
+    const double T = hmass + block_reduce_sum(tid < m ? d[tid] : 0.0, red);
+    const double Tn = ipow(T, n);
+    double ci = 1.0, rho = 0.5, wi = 1.0;
+    if (tid < m) {
+        sm.col[tid] = ipow(fmax(T - d[tid], 0.0), n);        // mass of tuples avoiding token tid
+        ci = Tn - sm.col[tid];
+        rho = fmin(rhs[tid] / ci, 1.0 - 1e-3);
+        wi = slack ? rho / (1.0 - rho) : rhs[tid] / d[tid];
+    }
+    if (!slack) {
+        const double ml = block_reduce_sum(tid < m ? log(wi) : 0.0, red) / (double)m;
+        wi *= exp(-ml);
+    }
+    if (tid < m) sm.w[tid] = wi;
+    __syncthreads();
+    // Pr[i and j drafted, all drafts inside] once, in the (still unused) contraction accumulator
+    for (int e = tid; e < m * kMP; e += kFT) {
+        const int i = e / kMP, j = e - i * kMP;
+        if (j < m) {
+            const double pij = Tn - sm.col[i] - sm.col[j] + ipow(fmax(T - d[i] - d[j], 0.0), n);
+            sm.Jacc[i * kJS + j] = (i == j) ? 0.f : (float)pij;
+        }
+    }
+    __syncthreads();
+    for (int sweep = 0; sweep < kFSweeps; sweep++) {
+        // S_i = sum_j Pr[i and j drafted] w_j / Pr[i drafted]: four rows per warp at a time (independent
+        // reductions interleave), lanes over j
+        for (int i0 = 4 * warp; i0 < m; i0 += 4 * kFW) {
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            for (int j = lane; j < m; j += 32) {
+                const double wj = sm.w[j];
+#pragma unroll
+                for (int a2 = 0; a2 < 4; a2++)
+                    if (i0 + a2 < m) acc[a2] = fma((double)sm.Jacc[(i0 + a2) * kJS + j], wj, acc[a2]);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int a2 = 0; a2 < 4; a2++) acc[a2] += __shfl_xor_sync(0xffffffffu, acc[a2], o);
+            }
+            if (lane < 4 && i0 + lane < m)
+                sm.delta[i0 + lane] = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
+        }
+        __syncthreads();
+        if (tid < m) {
+            const double Si = sm.delta[tid] / ci;
+            wi = rho / (1.0 - rho) * (slack ? 1.0 + Si : fmax(Si, 1e-300));
+        }
+        if (!slack) {
+            const double ml = block_reduce_sum(tid < m ? log(wi) : 0.0, red) / (double)m;
+            wi *= exp(-ml);
+        }
+        __syncthreads();
+        if (tid < m) sm.w[tid] = wi;
+        __syncthreads();
+    }
+    if (tid < m) sm.alpha[tid] = fmin(fmax(log(wi), -kFAlphaClamp), kFAlphaClamp);
+    __syncthreads();
+
+    int status = GR_NOT_CONVERGED, it = 0;
+    double rn = 0.0, rprev = 1.0e300, lam = 1.0;
+    for (; it < max_iters; it++) {
+        // far from the solution the trapezoid step is doubled (quadrature error ~4e-6, far below the gradient
+        // norm there): half the nodes, every one of them a Hessian node.  Convergence is only ever declared on
+        // the full grid.
+        const bool coarse = rprev > 1.0e-2;
+        fast_grid(sm, m, n, slack, coarse ? 2.0 * qstep : qstep);
+        // close to the solution the next point is expected to pass the test (quadratic convergence): evaluate
+        // the gradient alone first and add the Hessian only if the test fails after all
+        const bool expect_done = !coarse && it > 0 && lam == 1.0 && rprev * rprev * 30.0 < tol;
+        fast_eval<NT, TPL>(sm, m, n, d, hmass, !expect_done, coarse ? 1 : 2);
+        rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
+        if (rn <= tol && !coarse) { status = GR_OK; it++; break; }
+        if (expect_done) {
+            fast_eval<NT, TPL>(sm, m, n, d, hmass, true, 2);
+            it++;
+        }
+        if (!(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
+            // the last step did not reduce the gradient norm: retry it at half length
+            lam *= 0.5;
+            if (tid < m) sm.alpha[tid] = sm.alpha_prev[tid] + lam * sm.delta[tid];
+            __syncthreads();
+            continue;
+        }
+        rprev = rn; lam = 1.0;
+        if (tid < m) sm.alpha_prev[tid] = sm.alpha[tid];
+        if (tid == 0) sm.scal[SC_FAIL] = 0.0;
+        // Newton step with the Hessian (off-diagonal from the contraction, diagonal g - g2); an outer block's
+        // function is constant along (1,...,1): pin that direction with 1/m everywhere
+        fast_newton_step(sm, m, rhs, slack ? 0.0 : 1.0 / (double)m);
+        const bool fail = sm.scal[SC_FAIL] != 0.0;
+        if (fail) {
+            // proportional-fitting step  alpha += log(rhs / g)
+            if (tid < m) sm.delta[tid] = log(rhs[tid] / sm.g[tid]);
+            __syncthreads();
+        }
+        double dl = tid < m ? sm.delta[tid] : 0.0;
+        if (!(dl == dl)) dl = 0.0;
+        if (!slack) dl -= block_reduce_sum(tid < m ? dl : 0.0, red) / (double)m;
+        const double dm = block_reduce_max(tid < m ? fabs(dl) : 0.0, red);
+        // a full Newton step below 1e-11 in alpha: the weights cannot be improved at this quadrature accuracy
+        if (!fail && dm < 1.0e-11) { status = GR_OK; it++; break; }
+        if (dm > kFStepClamp) dl *= kFStepClamp / dm;
+        if (tid < m) {
+            sm.delta[tid] = dl;
+            sm.alpha[tid] = fmin(fmax(sm.alpha[tid] + dl, -kFAlphaClamp), kFAlphaClamp);
+        }
+        __syncthreads();
+    }
+    *gnorm = rn;
+    *iters = it;
+    return status;
+}
+
+template <int NT, int TPL>
+__global__ void __launch_bounds__(kFT, 3)
+fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
+                  double temp_t, double temp_d, double tol, int max_iters, double qstep,
+                  float* __restrict__ alpha_out, int* __restrict__ status_out)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int tid = threadIdx.x;
+    const long long b = blockIdx.x;
+    char* pb = params + (size_t)b * pstride;
+    ParamView pv = view_params(pb, kcap);
+    const WsView wv = view_ws(ws, b);
+    if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
+        if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
+        return;
+    }
+    const int KP = kcap;
+    FastLayout L(KP, NT);
+    double* base = reinterpret_cast<double*>(smem_raw);
+    FSm sm;
+    sm.d = base + L.d; sm.tg = base + L.tg; sm.p = base + L.p; sm.r = base + L.r; sm.key = base + L.key;
+    sm.psi = base + L.psi; sm.Dr = base + L.Dr; sm.alpha = base + L.alpha; sm.alpha_prev = base + L.alpha_prev;
+    sm.delta = base + L.delta; sm.w = base + L.w; sm.g = base + L.g; sm.g2 = base + L.g2; sm.col = base + L.col;
+    sm.gw = base + L.gw; sm.g2w = base + L.g2w; sm.tq = base + L.tq; sm.cq = base + L.cq; sm.scal = base + L.scal;
+    sm.J = base + L.uni;
+    sm.AS = reinterpret_cast<float*>(base + L.uni);
+    sm.HS = sm.AS + kJC * NT * kMS;
+    sm.Jacc = reinterpret_cast<float*>(smem_raw + L.jacc_bytes_off);
+    int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
+    sm.id = ib; sm.blk = ib + KP; sm.itmp = ib + 2 * KP;
+    sm.KP = KP;
+    PrepSm ps;
+    ps.d = sm.d; ps.tg = sm.tg; ps.p = sm.p; ps.r = sm.r; ps.key = sm.key; ps.psi = sm.psi; ps.Dr = sm.Dr;
+    ps.id = sm.id; ps.blk = sm.blk; ps.itmp = sm.itmp; ps.red = sm.scal + SC_RED; ps.out3 = sm.scal + 16;
+    const PrepResult pr = prep_instance(ps, wv, pv.h, V, n, topk, temp_t, temp_d);
+    const int k = pr.k, jstar = pr.jstar;
+
+    int status = GR_OK, iters_total = 0;
+    double gnorm_total = 0.0;
+    if (tid < k) pv.w[tid] = 1.0;
+    if (jstar > 0) {
+        double gn; int it;
+        const int st = fast_system<NT, TPL>(sm, jstar, n, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+        if (st != GR_OK) status = kNeedFallback;
+        gnorm_total += gn; iters_total += it;
+        if (tid < jstar) pv.w[tid] = sm.w[tid];
+        __syncthreads();
+    }
+    int lo = jstar;
+    while (lo < k && status == GR_OK) {
+        int hi = lo;
+        const int bk = sm.blk[lo];
+        while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
+        const int m = hi - lo + 1;
+        if (m >= 2) {
+            double gn; int it;
+            const int st = fast_system<NT, TPL>(sm, m, n, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep,
+                                                &gn, &it);
+            if (st != GR_OK) status = kNeedFallback;
+            gnorm_total += gn; iters_total += it;
+            if (tid < m) pv.w[lo + tid] = sm.w[tid];
+            __syncthreads();
+        }
+        lo = hi + 1;
+    }
+    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
+}
+
+template <int NT, int TPL>
+int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
+                         double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out,
+                         int* status_out, cudaStream_t st)
+{
+    const int smem = fast_smem_bytes(kcap, NT);
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 96 * 1024) != cudaSuccess)
+            return GR_E_LAUNCH;
+        configured = true;
+    }
+    fast_solve_kernel<NT, TPL><<<batch, kFT, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
+                                                         max_iters, qstep, alpha_out, status_out);
+    return GR_OK;
+}
+
+// One translation unit per series length instantiates its kernels (they compile in parallel).
+#define GR_FAST_ARGS                                                                                              \
+    const char *ws, char *params, int pstride, int kcap, int V, int n, int topk, double temp_t, double temp_d,   \
+        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, cudaStream_t st
+#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, st
+#define GR_FAST_INSTANTIATE(NT)                                                                \
+    int launch_fast_n##NT(GR_FAST_ARGS) {                                                       \
+        return kcap <= 32 ? launch_fast_t<NT, 1>(GR_FAST_PASS) : launch_fast_t<NT, 2>(GR_FAST_PASS); \
+    }
+
+}  // namespace gr
