@@ -25,10 +25,11 @@
 
 namespace gr {
 
-constexpr int kFT = 128;              // threads per CTA
+constexpr int kFT = 96;               // threads per CTA (at least kMP)
+constexpr int kFCtas = 4;             // CTAs per SM the kernels are compiled for
 constexpr int kFW = kFT / 32;         // warps per CTA
 constexpr int kMP = 64;               // padded support size of this kernel
-constexpr int kJC = 8;                // Hessian nodes staged per chunk
+constexpr int kJC = 6;                // Hessian nodes staged per chunk
 constexpr double kFTEnd = 25.0;       // quadrature range constants, identical to the robust kernel's
 constexpr double kFDrop = 1.0;
 constexpr double kFTail = 3.0;
@@ -37,7 +38,7 @@ constexpr int kMS = 72;               // row stride of the staged operands (floa
 constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
-constexpr int kFSweeps = 3;           // fixed-point sweeps of the mean-field start
+constexpr int kFSweeps = 5;           // fixed-point sweeps of the starting point
 
 struct FastLayout {
     int KP;
@@ -439,7 +440,7 @@ static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double 
 // Newton step: fp32 Cholesky of the Hessian in place in the contraction accumulator (row stride kJS),
 // with the forward substitution carried along and the backward substitution on warp 0.  The step only
 // steers the iteration (the fp64 gradient decides convergence) and the Hessian was accumulated in fp32.
-// Thread (ty, tx) = (tid / 8, tid % 8) updates the trailing rows j+1+ty+16a and columns j+1+tx+8b.
+// Thread (ty, tx) = (tid / 8, tid % 8) updates the trailing rows j+1+ty+(kFT/8)a and columns j+1+tx+8b.
 // Matrix: off-diagonal -Jacc (lower triangle), diagonal g - g2, plus `add` everywhere.  Writes the step
 // into sm.delta; sets SC_FAIL when a pivot is not positive.
 static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
@@ -456,7 +457,17 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
     }
     if (tid < m) {
         Jm[tid * kJS + tid] = (float)(sm.g[tid] - sm.g2[tid]) + addf;
-        yv[tid] = -(float)(sm.g[tid] - rhs[tid]);
+        // Right-hand side.  Along its own coordinate a token's flow behaves like a logistic curve
+        // g_i = c sigma(alpha_i - kappa): linear in w_i while the token is light, saturating at the flow c of the
+        // tuples it can win at all once it is heavy.  The curve through the current value and slope
+        // (H_ii = g_i (1 - g_i / c)  gives  c = g_i^2 / g2_i)  is inverted exactly:  H_ii (logit(rhs_i / c) -
+        // logit(g_i / c))  replaces  rhs_i - g_i.  Near the solution the two agree to first order; far from it a
+        // token close to saturation (weight in the thousands) is placed at once, where the plain residual moves
+        // its weight by a factor e per step, and a light token gets the multiplicative update log(rhs_i / g_i).
+        const double gi = sm.g[tid], g2i = sm.g2[tid], ri = rhs[tid];
+        const double den = gi * fmax(1.0 - ri * g2i / (gi * gi), 1e-3);
+        const double arg = fmax((ri - gi) / den, -1.0 + 1e-12);
+        yv[tid] = (float)((gi - g2i) * log1p(arg));
     }
     __syncthreads();
     bool bad = false;
@@ -528,7 +539,7 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
 #pragma unroll
             for (int c = 0; c < 4; c++) cl[b2][c] = (l < m && c < nb) ? Jm[l * kJS + j0 + c] : 0.f;
         }
-        for (int i = t0 + ty; i < m; i += 16) {
+        for (int i = t0 + ty; i < m; i += kFT / 8) {
             float* row = Jm + i * kJS;
             float ci[4];
 #pragma unroll
@@ -619,16 +630,32 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
         }
     }
     __syncthreads();
+    // Sweeps of  w_i = rho_i / (1 - rho_i) * (slack + S_i),  S_i = the weight token i is up against.  A competitor j,
+    // present with probability pi_ij = Pr[i and j drafted] / Pr[i drafted], adds to S_i the weight e_j for which
+    // 1 / (A + e_j) = (1 - pi_ij) / A + pi_ij / (A + w_j),  A = slack + w_i + S_i:  e_j = A pi_ij w_j / (A + w_j (1 - pi_ij)).
+    // For w_j << A this is the mean-field value pi_ij w_j; a huge w_j counts for A pi_ij / (1 - pi_ij) only (token i
+    // simply loses the tuples that contain j), which keeps the start sane when a few weights are in the thousands.
+    // fp32: it is a starting point.
+    if (tid < m) { sm.g2[tid] = 1.0 / ci; sm.g[tid] = (slack ? 1.0 : 0.0) + wi; }
+    __syncthreads();
     for (int sweep = 0; sweep < kFSweeps; sweep++) {
-        // S_i = sum_j Pr[i and j drafted] w_j / Pr[i drafted]: four rows per warp at a time (independent
-        // reductions interleave), lanes over j
+        // four rows per warp at a time (independent reductions interleave), lanes over j
         for (int i0 = 4 * warp; i0 < m; i0 += 4 * kFW) {
-            double acc[4] = {0.0, 0.0, 0.0, 0.0};
-            for (int j = lane; j < m; j += 32) {
-                const double wj = sm.w[j];
+            float acc[4] = {0.f, 0.f, 0.f, 0.f}, Ai[4], ic[4];
 #pragma unroll
-                for (int a2 = 0; a2 < 4; a2++)
-                    if (i0 + a2 < m) acc[a2] = fma((double)sm.Jacc[(i0 + a2) * kJS + j], wj, acc[a2]);
+            for (int a2 = 0; a2 < 4; a2++) {
+                const int i = min(i0 + a2, m - 1);
+                Ai[a2] = (float)sm.g[i]; ic[a2] = (float)sm.g2[i];
+            }
+            for (int j = lane; j < m; j += 32) {
+                const float wj = (float)sm.w[j];
+#pragma unroll
+                for (int a2 = 0; a2 < 4; a2++) {
+                    if (i0 + a2 < m) {
+                        const float pij = fminf(sm.Jacc[(i0 + a2) * kJS + j] * ic[a2], 1.f);
+                        acc[a2] += __fdividef(Ai[a2] * pij * wj, Ai[a2] + wj * (1.f - pij));
+                    }
+                }
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
@@ -636,26 +663,32 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
                 for (int a2 = 0; a2 < 4; a2++) acc[a2] += __shfl_xor_sync(0xffffffffu, acc[a2], o);
             }
             if (lane < 4 && i0 + lane < m)
-                sm.delta[i0 + lane] = lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3]));
+                sm.delta[i0 + lane] = (double)(lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3])));
         }
         __syncthreads();
+        double Si = 0.0;
         if (tid < m) {
-            const double Si = sm.delta[tid] / ci;
+            Si = sm.delta[tid];
             wi = rho / (1.0 - rho) * (slack ? 1.0 + Si : fmax(Si, 1e-300));
         }
+        double scale = 1.0;
         if (!slack) {
             const double ml = block_reduce_sum(tid < m ? log(wi) : 0.0, red) / (double)m;
-            wi *= exp(-ml);
+            scale = exp(-ml);
+            wi *= scale;
         }
         __syncthreads();
-        if (tid < m) sm.w[tid] = wi;
+        if (tid < m) { sm.w[tid] = wi; sm.g[tid] = (slack ? 1.0 : 0.0) + wi + scale * Si; }
         __syncthreads();
     }
-    if (tid < m) sm.alpha[tid] = fmin(fmax(log(wi), -kFAlphaClamp), kFAlphaClamp);
+    if (tid < m) {
+        sm.alpha[tid] = fmin(fmax(log(wi), -kFAlphaClamp), kFAlphaClamp);
+    }
     __syncthreads();
 
     int status = GR_NOT_CONVERGED, it = 0;
     double rn = 0.0, rprev = 1.0e300, lam = 1.0;
+    bool was_coarse = true;
     for (; it < max_iters; it++) {
         // far from the solution the trapezoid step is doubled (quadrature error ~4e-6, far below the gradient
         // norm there): half the nodes, every one of them a Hessian node.  Convergence is only ever declared on
@@ -672,13 +705,19 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
             fast_eval<NT, TPL>(sm, m, n, d, hmass, true, 2);
             it++;
         }
-        if (!(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
+        // (a residual on the full grid is not compared with the coarse grid's: they differ by the coarse quadrature error)
+        const bool comparable = coarse == was_coarse;
+        was_coarse = coarse;
+        if (comparable && !(rn < rprev) && lam > 1.0 / 64.0 && it > 0) {
             // the last step did not reduce the gradient norm: retry it at half length
             lam *= 0.5;
             if (tid < m) sm.alpha[tid] = sm.alpha_prev[tid] + lam * sm.delta[tid];
             __syncthreads();
             continue;
         }
+        // observed contraction  r_k = C r_{k-1}^2  of the last full step (same grid on both sides)
+        const double cq2 = (comparable && !coarse && it > 0 && lam == 1.0) ? rn / (rprev * rprev) : 1.0e300;
+        const bool contracting = cq2 * rprev < 0.1;
         rprev = rn; lam = 1.0;
         if (tid < m) sm.alpha_prev[tid] = sm.alpha[tid];
         if (tid == 0) sm.scal[SC_FAIL] = 0.0;
@@ -703,6 +742,15 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
             sm.alpha[tid] = fmin(fmax(sm.alpha[tid] + dl, -kFAlphaClamp), kFAlphaClamp);
         }
         __syncthreads();
+        // Newton has been contracting quadratically and the residual this step leaves behind, C r_k^2, is predicted
+        // ten times below the tolerance: take the step and stop without another evaluation
+        if (!fail && contracting && dm <= kFStepClamp && 10.0 * cq2 * rn * rn < tol) {
+            if (tid < m) sm.w[tid] = exp(sm.alpha[tid]);
+            __syncthreads();
+            rn = cq2 * rn * rn;
+            status = GR_OK; it++;
+            break;
+        }
     }
     *gnorm = rn;
     *iters = it;
@@ -710,7 +758,7 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
 }
 
 template <int NT, int TPL>
-__global__ void __launch_bounds__(kFT, 3)
+__global__ void __launch_bounds__(kFT, kFCtas)
 fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
                   double temp_t, double temp_d, double tol, int max_iters, double qstep,
                   float* __restrict__ alpha_out, int* __restrict__ status_out)
@@ -787,6 +835,10 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
     if (!configured) {
         if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  96 * 1024) != cudaSuccess)
+            return GR_E_LAUNCH;
+        // the CTAs are small: ask for the largest shared-memory carve-out so that kFCtas of them fit on an SM
+        if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                 cudaSharedmemCarveoutMaxShared) != cudaSuccess)
             return GR_E_LAUNCH;
         configured = true;
     }
