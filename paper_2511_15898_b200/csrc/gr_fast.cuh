@@ -440,12 +440,11 @@ static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double 
 // Newton step: fp32 Cholesky of the Hessian in place in the contraction accumulator (row stride kJS),
 // with the forward substitution carried along and the backward substitution on warp 0.  The step only
 // steers the iteration (the fp64 gradient decides convergence) and the Hessian was accumulated in fp32.
-// Thread (ty, tx) = (tid / 8, tid % 8) updates the trailing rows j+1+ty+(kFT/8)a and columns j+1+tx+8b.
 // Matrix: off-diagonal -Jacc (lower triangle), diagonal g - g2, plus `add` everywhere.  Writes the step
 // into sm.delta; sets SC_FAIL when a pivot is not positive.
 static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
 {
-    const int tid = threadIdx.x, ty = tid >> 3, tx = tid & 7;
+    const int tid = threadIdx.x;
     float* Jm = sm.Jacc;
     float* yv = reinterpret_cast<float*>(sm.J);        // [kMP] working right-hand side
     float* yf = yv + kMP;                              // [kMP] forward-substituted right-hand side, then the solution
@@ -471,7 +470,9 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
     }
     __syncthreads();
     bool bad = false;
-    // blocked right-looking factorisation, four columns per pair of barriers
+    // Blocked right-looking factorisation in panels of eight columns, each factored as two blocks of four.  After
+    // the first block only the panel's other four columns are brought up to date (one row per thread); after the
+    // second the rest of the matrix takes the panel's rank-8 update on the tensor cores.
     for (int j0 = 0; j0 < m; j0 += 4) {
         const int nb = min(4, m - j0);
         // every thread factors the diagonal block (at most 4 x 4) in registers
@@ -506,8 +507,8 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
         __syncthreads();                       // every thread has read the block before it is overwritten
         // panel below the block: one row per thread
         const int i1 = j0 + nb + tid;
+        float lp[4] = {0.f, 0.f, 0.f, 0.f};
         if (i1 < m) {
-            float lp[4];
             float yi = yv[i1];
 #pragma unroll
             for (int c = 0; c < 4; c++) {
@@ -532,26 +533,53 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
         __syncthreads();
         // trailing update  J[i][l] -= sum_c L[i][c] L[l][c],  j0 + nb <= l <= i
         const int t0 = j0 + nb;
-        float cl[8][4];
+        if ((j0 & 7) == 0) {
+            // first block of the panel: only the panel's own remaining columns, row i1 by its thread
+            if (i1 < m) {
 #pragma unroll
-        for (int b2 = 0; b2 < 8; b2++) {
-            const int l = t0 + tx + 8 * b2;
+                for (int b2 = 0; b2 < 4; b2++) {
+                    const int l = t0 + b2;
+                    if (l <= i1) {
+                        float v = Jm[i1 * kJS + l];
 #pragma unroll
-            for (int c = 0; c < 4; c++) cl[b2][c] = (l < m && c < nb) ? Jm[l * kJS + j0 + c] : 0.f;
-        }
-        for (int i = t0 + ty; i < m; i += kFT / 8) {
-            float* row = Jm + i * kJS;
-            float ci[4];
+                        for (int c = 0; c < 4; c++) v = fmaf(-lp[c], Jm[l * kJS + j0 + c], v);
+                        Jm[i1 * kJS + l] = v;
+                    }
+                }
+            }
+        } else if (t0 < m) {
+            // second block: rank-8 update of everything right of the panel (columns j0 - 4 .. j0 + 3 of L) as
+            // m16n8k8 MMAs on 16 x 8 tiles of the lower triangle, operands split into two tf32 parts (~fp32 products)
+            const int lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
+            const int pa = j0 - 4;
+            int t = 0;
+            for (int mi = 0; t0 + 16 * mi < m; mi++) {
+                for (int ni = 0; ni <= 2 * mi + 1 && t0 + 8 * ni < m; ni++, t++) {
+                    if (t % kFW != warp) continue;
+                    const int ra = t0 + 16 * mi + gid, rb = ra + 8, l0 = t0 + 8 * ni, cb = l0 + gid;
+                    const bool oa = ra < m, ob = rb < m, oc = cb < m;
+                    const float fa[4] = {oa ? -Jm[ra * kJS + pa + tig] : 0.f, ob ? -Jm[rb * kJS + pa + tig] : 0.f,
+                                         oa ? -Jm[ra * kJS + pa + tig + 4] : 0.f, ob ? -Jm[rb * kJS + pa + tig + 4] : 0.f};
+                    const float fb[2] = {oc ? Jm[cb * kJS + pa + tig] : 0.f, oc ? Jm[cb * kJS + pa + tig + 4] : 0.f};
+                    float* C0 = Jm + ra * kJS + l0 + 2 * tig;
+                    float* C1 = Jm + rb * kJS + l0 + 2 * tig;
+                    float c0 = oa ? C0[0] : 0.f, c1 = oa ? C0[1] : 0.f, c2 = ob ? C1[0] : 0.f, c3 = ob ? C1[1] : 0.f;
+                    uint32_t ah[4], al[4], bh[2], bl[2];
 #pragma unroll
-            for (int c = 0; c < 4; c++) ci[c] = (c < nb) ? row[j0 + c] : 0.f;
+                    for (int z = 0; z < 4; z++) {
+                        const float hi = to_tf32(fa[z]);
+                        ah[z] = __float_as_uint(hi); al[z] = __float_as_uint(to_tf32(fa[z] - hi));
+                    }
 #pragma unroll
-            for (int b2 = 0; b2 < 8; b2++) {
-                const int l = t0 + tx + 8 * b2;
-                if (l <= i) {
-                    float v = row[l];
-#pragma unroll
-                    for (int c = 0; c < 4; c++) v = fmaf(-ci[c], cl[b2][c], v);
-                    row[l] = v;
+                    for (int z = 0; z < 2; z++) {
+                        const float hi = to_tf32(fb[z]);
+                        bh[z] = __float_as_uint(hi); bl[z] = __float_as_uint(to_tf32(fb[z] - hi));
+                    }
+                    mma_tf32(c0, c1, c2, c3, al[0], al[1], al[2], al[3], bh[0], bh[1]);
+                    mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bl[0], bl[1]);
+                    mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bh[0], bh[1]);
+                    if (oa) { C0[0] = c0; C0[1] = c1; }
+                    if (ob) { C1[0] = c2; C1[1] = c3; }
                 }
             }
         }
@@ -562,35 +590,26 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
         __syncthreads();
         return;
     }
-    // backward substitution L^T x = y on warp 0, four unknowns at a time: every lane solves the 4 x 4
-    // triangle redundantly, then the lanes update the unknowns above it
+    // backward substitution L^T x = y on warp 0, column-oriented with the right-hand side in registers (lane l holds
+    // entries l and l + 32): unknown e is finished by its owner, broadcast, and taken out of the entries above it.
+    // One multiply, one shuffle and one FMA per unknown on the critical path; row e of L is fetched one step ahead.
     if (tid < 32) {
-        for (int e0 = ((m - 1) >> 2) << 2; e0 >= 0; e0 -= 4) {
-            const int nb = min(4, m - e0);
-            float x[4];
-#pragma unroll
-            for (int c = 3; c >= 0; c--) {
-                float v = 0.f;
-                if (c < nb) {
-                    v = yf[e0 + c];
-#pragma unroll
-                    for (int c2 = 3; c2 > c; c2--)
-                        if (c2 < nb) v = fmaf(-Jm[(e0 + c2) * kJS + e0 + c], x[c2], v);
-                    v = v / dg[e0 + c];
-                }
-                x[c] = v;
+        const int lane = tid;
+        float y0 = lane < m ? yf[lane] : 0.f, y1 = lane + 32 < m ? yf[lane + 32] : 0.f;
+        const float r0 = lane < m ? 1.f / dg[lane] : 0.f, r1 = lane + 32 < m ? 1.f / dg[lane + 32] : 0.f;
+        float a0n = Jm[(m - 1) * kJS + lane], a1n = Jm[(m - 1) * kJS + lane + 32];
+        for (int e = m - 1; e >= 0; e--) {
+            const float a0 = a0n, a1 = a1n;
+            if (e > 0) { a0n = Jm[(e - 1) * kJS + lane]; a1n = Jm[(e - 1) * kJS + lane + 32]; }
+            const float xe = __shfl_sync(0xffffffffu, (e & 32) ? y1 * r1 : y0 * r0, e & 31);
+            if (lane == (e & 31)) {
+                if (e & 32) y1 = xe; else y0 = xe;
             }
-            __syncwarp();
-            if (tid < nb) yf[e0 + tid] = tid == 0 ? x[0] : (tid == 1 ? x[1] : (tid == 2 ? x[2] : x[3]));
-            for (int l = tid; l < e0; l += 32) {
-                float v = yf[l];
-#pragma unroll
-                for (int c = 0; c < 4; c++)
-                    if (c < nb) v = fmaf(-Jm[(e0 + c) * kJS + l], x[c], v);
-                yf[l] = v;
-            }
-            __syncwarp();
+            if (lane < e) y0 = fmaf(-a0, xe, y0);
+            if (lane + 32 < e) y1 = fmaf(-a1, xe, y1);
         }
+        if (lane < m) yf[lane] = y0;
+        if (lane + 32 < m) yf[lane + 32] = y1;
     }
     __syncthreads();
     if (tid < m) sm.delta[tid] = (double)yf[tid];
@@ -638,37 +657,43 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     // fp32: it is a starting point.
     if (tid < m) { sm.g2[tid] = 1.0 / ci; sm.g[tid] = (slack ? 1.0 : 0.0) + wi; }
     __syncthreads();
+    float* part = sm.AS;                              // [kFW][kMP] partial sums (the staging area is idle here)
     for (int sweep = 0; sweep < kFSweeps; sweep++) {
-        // four rows per warp at a time (independent reductions interleave), lanes over j
-        for (int i0 = 4 * warp; i0 < m; i0 += 4 * kFW) {
-            float acc[4] = {0.f, 0.f, 0.f, 0.f}, Ai[4], ic[4];
-#pragma unroll
-            for (int a2 = 0; a2 < 4; a2++) {
-                const int i = min(i0 + a2, m - 1);
-                Ai[a2] = (float)sm.g[i]; ic[a2] = (float)sm.g2[i];
+        // lane = row (and row + 32), warp = a contiguous share of the columns: no shuffles, four independent sums
+        {
+            const int chunk = (m + kFW - 1) / kFW;
+            const int jlo = warp * chunk, jhi = min(m, jlo + chunk);
+            const int r0 = lane, r1 = lane + 32;
+            const bool on0 = r0 < m, on1 = r1 < m;
+            const float A0 = on0 ? (float)sm.g[r0] : 1.f, c0 = on0 ? (float)sm.g2[r0] : 0.f;
+            const float A1 = on1 ? (float)sm.g[r1] : 1.f, c1 = on1 ? (float)sm.g2[r1] : 0.f;
+            const float* row0 = sm.Jacc + (on0 ? r0 : 0) * kJS;
+            const float* row1 = sm.Jacc + (on1 ? r1 : 0) * kJS;
+            float s0a = 0.f, s0b = 0.f, s1a = 0.f, s1b = 0.f;
+            int j = jlo;
+            for (; j + 1 < jhi; j += 2) {
+                const float wa = (float)sm.w[j], wb = (float)sm.w[j + 1];
+                const float p0a = fminf(row0[j] * c0, 1.f), p0b = fminf(row0[j + 1] * c0, 1.f);
+                const float p1a = fminf(row1[j] * c1, 1.f), p1b = fminf(row1[j + 1] * c1, 1.f);
+                s0a += __fdividef(A0 * p0a * wa, A0 + wa * (1.f - p0a));
+                s0b += __fdividef(A0 * p0b * wb, A0 + wb * (1.f - p0b));
+                s1a += __fdividef(A1 * p1a * wa, A1 + wa * (1.f - p1a));
+                s1b += __fdividef(A1 * p1b * wb, A1 + wb * (1.f - p1b));
             }
-            for (int j = lane; j < m; j += 32) {
-                const float wj = (float)sm.w[j];
-#pragma unroll
-                for (int a2 = 0; a2 < 4; a2++) {
-                    if (i0 + a2 < m) {
-                        const float pij = fminf(sm.Jacc[(i0 + a2) * kJS + j] * ic[a2], 1.f);
-                        acc[a2] += __fdividef(Ai[a2] * pij * wj, Ai[a2] + wj * (1.f - pij));
-                    }
-                }
+            if (j < jhi) {
+                const float wa = (float)sm.w[j];
+                const float p0a = fminf(row0[j] * c0, 1.f), p1a = fminf(row1[j] * c1, 1.f);
+                s0a += __fdividef(A0 * p0a * wa, A0 + wa * (1.f - p0a));
+                s1a += __fdividef(A1 * p1a * wa, A1 + wa * (1.f - p1a));
             }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-                for (int a2 = 0; a2 < 4; a2++) acc[a2] += __shfl_xor_sync(0xffffffffu, acc[a2], o);
-            }
-            if (lane < 4 && i0 + lane < m)
-                sm.delta[i0 + lane] = (double)(lane == 0 ? acc[0] : (lane == 1 ? acc[1] : (lane == 2 ? acc[2] : acc[3])));
+            part[warp * kMP + r0] = s0a + s0b;
+            part[warp * kMP + r1] = s1a + s1b;
         }
         __syncthreads();
         double Si = 0.0;
         if (tid < m) {
-            Si = sm.delta[tid];
+#pragma unroll
+            for (int w2 = 0; w2 < kFW; w2++) Si += (double)part[w2 * kMP + tid];
             wi = rho / (1.0 - rho) * (slack ? 1.0 + Si : fmax(Si, 1e-300));
         }
         double scale = 1.0;
