@@ -470,59 +470,57 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
     }
     __syncthreads();
     bool bad = false;
-    // Blocked right-looking factorisation in panels of eight columns, each factored as two blocks of four.  After
-    // the first block only the panel's other four columns are brought up to date (one row per thread); after the
-    // second the rest of the matrix takes the panel's rank-8 update on the tensor cores.
-    for (int j0 = 0; j0 < m; j0 += 4) {
-        const int nb = min(4, m - j0);
-        // every thread factors the diagonal block (at most 4 x 4) in registers
-        float Lb[4][4], yb[4], dinv[4];
+    // Blocked right-looking factorisation in panels of eight columns: every thread factors the 8 x 8 diagonal block
+    // in registers (redundantly: no exchange needed), one thread per row solves the panel below it and carries the
+    // forward substitution along, and the rest of the matrix takes the panel's rank-8 update on the tensor cores.
+    for (int j0 = 0; j0 < m; j0 += 8) {
+        const int nb = min(8, m - j0);
+        float Lb[8][8], yb[8], dinv[8];
 #pragma unroll
-        for (int c = 0; c < 4; c++) {
+        for (int c = 0; c < 8; c++) {
 #pragma unroll
             for (int c2 = 0; c2 <= c; c2++) Lb[c][c2] = (c < nb) ? Jm[(j0 + c) * kJS + j0 + c2] : (c == c2 ? 1.f : 0.f);
             yb[c] = (c < nb) ? yv[j0 + c] : 0.f;
         }
 #pragma unroll
-        for (int c = 0; c < 4; c++) {
-            float dv = Lb[c][c];
-#pragma unroll
-            for (int e2 = 0; e2 < c; e2++) dv = fmaf(-Lb[c][e2], Lb[c][e2], dv);
+        for (int c = 0; c < 8; c++) {
+            const float dv = Lb[c][c];
             if (!(dv > 0.f)) bad = true;
             dinv[c] = rsqrtf(dv);
             Lb[c][c] = dv * dinv[c];
-            float yc = yb[c];
+            yb[c] *= dinv[c];
 #pragma unroll
-            for (int e2 = 0; e2 < c; e2++) yc = fmaf(-Lb[c][e2], yb[e2], yc);
-            yb[c] = yc * dinv[c];
+            for (int r2 = c + 1; r2 < 8; r2++) Lb[r2][c] *= dinv[c];
 #pragma unroll
-            for (int r2 = c + 1; r2 < 4; r2++) {
-                float v = Lb[r2][c];
+            for (int r2 = c + 1; r2 < 8; r2++) {
 #pragma unroll
-                for (int e2 = 0; e2 < c; e2++) v = fmaf(-Lb[r2][e2], Lb[c][e2], v);
-                Lb[r2][c] = v * dinv[c];
+                for (int c3 = c + 1; c3 <= r2; c3++) Lb[r2][c3] = fmaf(-Lb[r2][c], Lb[c3][c], Lb[r2][c3]);
+                yb[r2] = fmaf(-Lb[r2][c], yb[c], yb[r2]);
             }
         }
         if (bad) break;
-        __syncthreads();                       // every thread has read the block before it is overwritten
-        // panel below the block: one row per thread
+        // panel below the block: one row per thread (it touches no entry of the block itself)
         const int i1 = j0 + nb + tid;
-        float lp[4] = {0.f, 0.f, 0.f, 0.f};
         if (i1 < m) {
+            float v[8];
+#pragma unroll
+            for (int c = 0; c < 8; c++) v[c] = (c < nb) ? Jm[i1 * kJS + j0 + c] : 0.f;
             float yi = yv[i1];
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
-                float v = (c < nb) ? Jm[i1 * kJS + j0 + c] : 0.f;
+            for (int c = 0; c < 8; c++) {
+                const float lc = v[c] * dinv[c];
 #pragma unroll
-                for (int e2 = 0; e2 < c; e2++) v = fmaf(-lp[e2], Lb[c][e2], v);
-                lp[c] = v * dinv[c];
-                if (c < nb) { Jm[i1 * kJS + j0 + c] = lp[c]; yi = fmaf(-lp[c], yb[c], yi); }
+                for (int c3 = c + 1; c3 < 8; c3++) v[c3] = fmaf(-lc, Lb[c3][c], v[c3]);
+                yi = fmaf(-lc, yb[c], yi);
+                if (c < nb) Jm[i1 * kJS + j0 + c] = lc;
             }
             yv[i1] = yi;
         }
+        __syncthreads();
+        // every thread has read the block by now: one of them stores its factor
         if (tid == kFT - 1) {
 #pragma unroll
-            for (int c = 0; c < 4; c++) {
+            for (int c = 0; c < 8; c++) {
                 if (c < nb) {
                     dg[j0 + c] = Lb[c][c]; yf[j0 + c] = yb[c];
 #pragma unroll
@@ -530,37 +528,20 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
                 }
             }
         }
-        __syncthreads();
-        // trailing update  J[i][l] -= sum_c L[i][c] L[l][c],  j0 + nb <= l <= i
-        const int t0 = j0 + nb;
-        if ((j0 & 7) == 0) {
-            // first block of the panel: only the panel's own remaining columns, row i1 by its thread
-            if (i1 < m) {
-#pragma unroll
-                for (int b2 = 0; b2 < 4; b2++) {
-                    const int l = t0 + b2;
-                    if (l <= i1) {
-                        float v = Jm[i1 * kJS + l];
-#pragma unroll
-                        for (int c = 0; c < 4; c++) v = fmaf(-lp[c], Jm[l * kJS + j0 + c], v);
-                        Jm[i1 * kJS + l] = v;
-                    }
-                }
-            }
-        } else if (t0 < m) {
-            // second block: rank-8 update of everything right of the panel (columns j0 - 4 .. j0 + 3 of L) as
-            // m16n8k8 MMAs on 16 x 8 tiles of the lower triangle, operands split into two tf32 parts (~fp32 products)
+        // trailing update  J[i][l] -= sum_c L[i][c] L[l][c],  j0 + 8 <= l <= i:  m16n8k8 MMAs on the 16 x 8 tiles of
+        // the lower triangle, operands split into two tf32 parts (~fp32 products)
+        const int t0 = j0 + 8;
+        if (t0 < m) {
             const int lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
-            const int pa = j0 - 4;
             int t = 0;
             for (int mi = 0; t0 + 16 * mi < m; mi++) {
                 for (int ni = 0; ni <= 2 * mi + 1 && t0 + 8 * ni < m; ni++, t++) {
                     if (t % kFW != warp) continue;
                     const int ra = t0 + 16 * mi + gid, rb = ra + 8, l0 = t0 + 8 * ni, cb = l0 + gid;
                     const bool oa = ra < m, ob = rb < m, oc = cb < m;
-                    const float fa[4] = {oa ? -Jm[ra * kJS + pa + tig] : 0.f, ob ? -Jm[rb * kJS + pa + tig] : 0.f,
-                                         oa ? -Jm[ra * kJS + pa + tig + 4] : 0.f, ob ? -Jm[rb * kJS + pa + tig + 4] : 0.f};
-                    const float fb[2] = {oc ? Jm[cb * kJS + pa + tig] : 0.f, oc ? Jm[cb * kJS + pa + tig + 4] : 0.f};
+                    const float fa[4] = {oa ? -Jm[ra * kJS + j0 + tig] : 0.f, ob ? -Jm[rb * kJS + j0 + tig] : 0.f,
+                                         oa ? -Jm[ra * kJS + j0 + tig + 4] : 0.f, ob ? -Jm[rb * kJS + j0 + tig + 4] : 0.f};
+                    const float fb[2] = {oc ? Jm[cb * kJS + j0 + tig] : 0.f, oc ? Jm[cb * kJS + j0 + tig + 4] : 0.f};
                     float* C0 = Jm + ra * kJS + l0 + 2 * tig;
                     float* C1 = Jm + rb * kJS + l0 + 2 * tig;
                     float c0 = oa ? C0[0] : 0.f, c1 = oa ? C0[1] : 0.f, c2 = ob ? C1[0] : 0.f, c3 = ob ? C1[1] : 0.f;
@@ -575,11 +556,13 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
                         const float hi = to_tf32(fb[z]);
                         bh[z] = __float_as_uint(hi); bl[z] = __float_as_uint(to_tf32(fb[z] - hi));
                     }
-                    mma_tf32(c0, c1, c2, c3, al[0], al[1], al[2], al[3], bh[0], bh[1]);
-                    mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bl[0], bl[1]);
+                    // three independent accumulations (the small cross terms apart), summed afterwards
+                    float e0 = 0.f, e1 = 0.f, e2 = 0.f, e3 = 0.f, f0 = 0.f, f1 = 0.f, f2 = 0.f, f3 = 0.f;
+                    mma_tf32(e0, e1, e2, e3, al[0], al[1], al[2], al[3], bh[0], bh[1]);
+                    mma_tf32(f0, f1, f2, f3, ah[0], ah[1], ah[2], ah[3], bl[0], bl[1]);
                     mma_tf32(c0, c1, c2, c3, ah[0], ah[1], ah[2], ah[3], bh[0], bh[1]);
-                    if (oa) { C0[0] = c0; C0[1] = c1; }
-                    if (ob) { C1[0] = c2; C1[1] = c3; }
+                    if (oa) { C0[0] = c0 + (e0 + f0); C0[1] = c1 + (e1 + f1); }
+                    if (ob) { C1[0] = c2 + (e2 + f2); C1[1] = c3 + (e3 + f3); }
                 }
             }
         }
@@ -720,16 +703,9 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
         // the full grid.
         const bool coarse = rprev > 1.0e-2;
         fast_grid(sm, m, n, slack, coarse ? 2.0 * qstep : qstep);
-        // close to the solution the next point is expected to pass the test (quadratic convergence): evaluate
-        // the gradient alone first and add the Hessian only if the test fails after all
-        const bool expect_done = !coarse && it > 0 && lam == 1.0 && rprev * rprev * 30.0 < tol;
-        fast_eval<NT, TPL>(sm, m, n, d, hmass, !expect_done, coarse ? 1 : 2);
+        fast_eval<NT, TPL>(sm, m, n, d, hmass, true, coarse ? 1 : 2);
         rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
         if (rn <= tol && !coarse) { status = GR_OK; it++; break; }
-        if (expect_done) {
-            fast_eval<NT, TPL>(sm, m, n, d, hmass, true, 2);
-            it++;
-        }
         // (a residual on the full grid is not compared with the coarse grid's: they differ by the coarse quadrature error)
         const bool comparable = coarse == was_coarse;
         was_coarse = coarse;

@@ -106,38 +106,69 @@ __device__ inline PrepResult prep_instance(const PrepSm& sm, const WsView& wv, H
     __syncthreads();
     // ---- prefix sums in order, psi along the chain, H* and alpha* (Eq. "subset-select")
     if (tid == 0) {
+        // (summed in order, one after the other, four loads ahead of the stores)
         double Tg = 0.0, Dr = 0.0;
         sm.psi[0] = 0.0; sm.Dr[0] = 0.0;
-        for (int j = 1; j <= k; j++) {
-            Tg += sm.tg[j - 1]; Dr += sm.d[j - 1];
-            if (j == k) { Dr = 1.0; if (kfull == V) Tg = 1.0; }   // both distributions are normalised
-            sm.psi[j] = Tg; sm.Dr[j] = Dr;
+        for (int j0 = 0; j0 < k; j0 += 4) {
+            double tv[4], dv[4];
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const bool in = j0 + u < k;
+                tv[u] = in ? sm.tg[j0 + u] : 0.0; dv[u] = in ? sm.d[j0 + u] : 0.0;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; u++) {
+                const int j = j0 + u + 1;
+                if (j <= k) {
+                    Tg += tv[u]; Dr += dv[u];
+                    if (j == k) { Dr = 1.0; if (kfull == V) Tg = 1.0; }   // both distributions are normalised
+                    sm.psi[j] = Tg; sm.Dr[j] = Dr;
+                }
+            }
         }
     }
     __syncthreads();
-    for (int j = 1 + tid; j <= k; j += blockDim.x) sm.psi[j] = sm.psi[j] - pow(sm.Dr[j], (double)n);
+    for (int j = 1 + tid; j <= k; j += blockDim.x) {
+        const double base = sm.Dr[j];
+        double pw = 1.0, sq = base;
+        for (int e = n; e > 0; e >>= 1) { if (e & 1) pw *= sq; sq *= sq; }
+        sm.psi[j] = sm.psi[j] - pw;
+    }
     __syncthreads();
-    if (tid == 0) {
-        int jstar = 0; double best = 0.0;
-        for (int j = 1; j <= k; j++) if (sm.psi[j] < best) { best = sm.psi[j]; jstar = j; }
-        // ---- outer residuals by cumulative minima along the increasing-ratio chain; blocks end at
-        //      every new strict minimum (Sec. 6.1, Thm "polymatroid", Lemma "q-convex")
-        for (int j = 0; j < jstar; j++) { sm.p[j] = sm.tg[j]; sm.r[j] = 0.0; sm.blk[j] = -1; }
-        double m_prev = sm.psi[k];
-        int blk = 0, open = 0;
-        for (int s = 1; s <= k - jstar; s++) {
-            const int pos = k - s;
-            const double c = sm.psi[k - s];
-            const bool record = c < m_prev;
-            const double mm = record ? c : m_prev;
-            sm.r[pos] = m_prev - mm;
-            sm.p[pos] = sm.tg[pos] - sm.r[pos];
-            sm.blk[pos] = blk; open = 1;
-            if (record) { blk++; open = 0; }
-            m_prev = mm;
+    // first strict minimum of psi (H* = the prefix up to it), every thread for itself
+    int jstar = 0; double best = 0.0;
+    for (int j = 1; j <= k; j++) {
+        const double v = sm.psi[j];
+        if (v < best) { best = v; jstar = j; }
+    }
+    // ---- outer residuals by cumulative minima along the increasing-ratio chain; blocks end at
+    //      every new strict minimum (Sec. 6.1, Thm "polymatroid", Lemma "q-convex").  One position per thread:
+    //      the running minimum that reaches a position is the minimum of psi over the positions above it
+    //      (exact in any order), and its block number counts the strict minima above it.
+    for (int pos = tid; pos < k; pos += blockDim.x) {
+        if (pos < jstar) {
+            sm.p[pos] = sm.tg[pos]; sm.r[pos] = 0.0; sm.blk[pos] = -1;
+        } else {
+            double m_prev = sm.psi[k];
+            int blk = 0;
+            for (int j = k - 1; j > pos; j--) {
+                const double c = sm.psi[j];
+                if (c < m_prev) { m_prev = c; blk++; }
+            }
+            const double c = sm.psi[pos];
+            const double rr = c < m_prev ? m_prev - c : 0.0;
+            sm.r[pos] = rr;
+            sm.p[pos] = sm.tg[pos] - rr;
+            sm.blk[pos] = blk;
+            if (pos == jstar) {
+                // the lowest position of the chain closes the last block: it is open unless this position is a record
+                sm.out3[1] = (double)(blk + 1);
+            }
         }
+    }
+    if (tid == 0) {
         sm.out3[0] = (double)jstar;
-        sm.out3[1] = (double)(blk + open);
+        if (jstar >= k) sm.out3[1] = 0.0;
         sm.out3[2] = 1.0 + best;
     }
     __syncthreads();
