@@ -61,6 +61,10 @@ extern "C" {
  *   tol        stop when the L1 norm of the gradient of the convex function
  *              (Theta for the inner system, Phi restricted to a block for the outer
  *              system; Sec. 6.2) is <= tol.                      default 1e-9
+ *              The faster kernel also stops after a Newton step whose predecessor
+ *              contracted quadratically (r_k = C r_{k-1}^2, C r_{k-1} < 0.1) when the
+ *              residual it leaves, C r_k^2, is predicted below tol / 10; the
+ *              reported gradient norm is then that prediction.
  *   max_iters  cap on gradient evaluations per system.            default 40
  *   quad_step  step of the trapezoid rule in the log-time variable used to
  *              evaluate the gradient integral; smaller is more accurate and
