@@ -44,6 +44,8 @@ extern "C" {
 #define GR_BAD_LOGITS            3  /* a NaN or infinite logit in the row                                 */
 #define GR_DRAFT_OUT_OF_SUPPORT  4  /* a drafted token does not belong to the draft support               */
 #define GR_STALE_PARAMS          5  /* params block was not written by gr_solve for this shape            */
+#define GR_PARTIAL_RULE          6  /* params written by gr_solve_verify: only the system its drafted tuple
+                                       selects was solved; gr_verify refuses such a block (token -1)       */
 
 /* host-side argument errors (return values) */
 #define GR_E_INVALID   (-1)  /* a size, temperature or option is out of range */
@@ -183,6 +185,24 @@ int gr_solve_static(const void* q_logits, const void* p_logits, int dtype, int V
  */
 int gr_verify(const void* params, const int* draft_tokens, const float* uniforms, int batch,
               int* out_token, unsigned char* out_accepted, int* status, void* stream);
+
+/*
+ * gr_solve_verify -- gr_solve and gr_verify in one call for drafts known beforehand:
+ * the solve kernel of every instance looks at its drafted tuple, solves only the
+ * system that tuple selects (Eq. "cases": the inner system when every drafted token
+ * lies in H*, else the lowest-ratio outer block the tuple meets; Algorithm 1 does the
+ * same) and finishes with the draw itself, so no separate verification launch and no
+ * second read of the rule.  Arguments as for gr_solve and gr_verify; `status` holds
+ * what gr_verify would report.  alpha_star is written as by gr_solve.  The params block
+ * is still written (for gr_read_rule); instances where a system was skipped carry
+ * GR_PARTIAL_RULE in it and must not be given to gr_verify with other drafts.
+ * Same return values as gr_solve.
+ */
+int gr_solve_verify(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk,
+                    float temp_target, float temp_draft, int batch, const gr_options* opt,
+                    const int* draft_tokens, const float* uniforms, void* params, void* workspace,
+                    float* alpha_star, int* out_token, unsigned char* out_accepted, int* status,
+                    void* stream);
 
 /*
  * gr_read_rule -- copies the rule of every instance out of `params` into plain

@@ -11,7 +11,7 @@ from __future__ import annotations
 import ctypes as C
 import dataclasses
 import os
-from typing import Optional
+from typing import Optional, Tuple
 
 import torch
 
@@ -19,6 +19,7 @@ GR_F32, GR_BF16 = 0, 1
 GR_OK, GR_NOT_CONVERGED, GR_SUPPORT_TOO_LARGE, GR_BAD_LOGITS, GR_DRAFT_OUT_OF_SUPPORT, GR_STALE_PARAMS = range(6)
 GR_MAX_SUPPORT, GR_MAX_DRAFTS = 128, 32
 GR_STATIC_MAX_BATCH = 256
+GR_PARTIAL_RULE = 6
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgr_b200.so")
@@ -61,6 +62,9 @@ def load_library():
     lib.gr_solve_static.restype = C.c_int
     lib.gr_solve_static.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int,
                                     C.POINTER(Options), vp, fp, ip, vp]
+    lib.gr_solve_verify.restype = C.c_int
+    lib.gr_solve_verify.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int,
+                                    C.POINTER(Options), ip, fp, vp, vp, fp, ip, vp, ip, vp]
     lib.gr_verify.restype = C.c_int
     lib.gr_verify.argtypes = [vp, ip, fp, C.c_int, ip, vp, ip, vp]
     lib.gr_read_rule.restype = C.c_int
@@ -101,6 +105,15 @@ def gr_solve_static(q_logits: int, p_logits: int, dtype: int, V: int, n: int, to
     return int(load_library().gr_solve_static(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch,
                                               C.byref(opt) if opt is not None else None, params, alpha_star, status,
                                               stream))
+
+
+def gr_solve_verify(q_logits: int, p_logits: int, dtype: int, V: int, n: int, topk: int, temp_target: float,
+                    temp_draft: float, batch: int, opt: Optional[Options], draft_tokens: int, uniforms: int,
+                    params: int, workspace: int, alpha_star: int, out_token: int, out_accepted: int, status: int,
+                    stream: int) -> int:
+    return int(load_library().gr_solve_verify(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch,
+                                              C.byref(opt) if opt is not None else None, draft_tokens, uniforms,
+                                              params, workspace, alpha_star, out_token, out_accepted, status, stream))
 
 
 def gr_verify(params: int, draft_tokens: int, uniforms: int, batch: int, out_token: int, out_accepted: int,
@@ -203,6 +216,46 @@ def verify(solved: Solved, draft_tokens: torch.Tensor, uniforms: torch.Tensor,
                    out.accepted.data_ptr(), out.status.data_ptr(), _stream())
     _check(rc, "gr_verify")
     return out
+
+
+def solve_verify(q_logits: torch.Tensor, p_logits: torch.Tensor, draft_tokens: torch.Tensor, uniforms: torch.Tensor,
+                 topk: int, temp_target: float = 1.0, temp_draft: float = 1.0, opt: Optional[Options] = None,
+                 out: Optional[Tuple[Solved, Verified]] = None) -> Tuple[Solved, Verified]:
+    """gr_solve_verify on torch CUDA tensors: one call, the solve kernel finishes every instance with its draw.
+    The returned Solved carries alpha* and the params block (partial where a system was skipped); the Verified's
+    status is what gr_verify would report."""
+    _need_cuda(q_logits, p_logits, draft_tokens, uniforms)
+    if q_logits.shape != p_logits.shape or q_logits.dim() != 2 or q_logits.dtype != p_logits.dtype:
+        raise GrError("q_logits and p_logits must be [B, V] tensors of one dtype")
+    B, V = q_logits.shape
+    if draft_tokens.dim() != 2 or draft_tokens.shape[0] != B or draft_tokens.dtype != torch.int32:
+        raise GrError("draft_tokens must be [B, n] int32")
+    n = int(draft_tokens.shape[1])
+    if uniforms.shape != (B, 2) or uniforms.dtype != torch.float32:
+        raise GrError("uniforms must be [B, 2] float32")
+    dev = q_logits.device
+    sv, vf = out if out is not None else (None, None)
+    if sv is None or sv.batch != B or sv.V != V or sv.n != n or sv.topk != topk:
+        pbytes = gr_params_bytes(V, n, topk, B)
+        wbytes = gr_workspace_bytes(V, n, topk, B)
+        if pbytes == 0 or wbytes == 0:
+            raise GrError("invalid shape")
+        sv = Solved(V, n, topk, B, torch.empty(pbytes, dtype=torch.uint8, device=dev),
+                    torch.empty(wbytes, dtype=torch.uint8, device=dev),
+                    torch.empty(B, dtype=torch.float32, device=dev),
+                    torch.empty(B, dtype=torch.int32, device=dev), q_logits)
+        vf = None
+    if vf is None or vf.token.shape[0] != B:
+        vf = Verified(torch.empty(B, dtype=torch.int32, device=dev), torch.empty(B, dtype=torch.uint8, device=dev),
+                      sv.status)
+    sv.q_logits = q_logits
+    vf.status = sv.status
+    rc = gr_solve_verify(q_logits.data_ptr(), p_logits.data_ptr(), _dtype_code(q_logits), V, n, topk, temp_target,
+                         temp_draft, B, opt, draft_tokens.data_ptr(), uniforms.data_ptr(), sv.params.data_ptr(),
+                         sv.workspace.data_ptr(), sv.alpha_star.data_ptr(), vf.token.data_ptr(),
+                         vf.accepted.data_ptr(), sv.status.data_ptr(), _stream())
+    _check(rc, "gr_solve_verify")
+    return sv, vf
 
 
 @dataclasses.dataclass

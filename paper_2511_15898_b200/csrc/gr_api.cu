@@ -1,16 +1,16 @@
 // Host side of the C interface declared in gr.h: argument checks and kernel launches.
 #include <math.h>
-#include "gr_common.cuh"
+#include "gr_verify.cuh"
 
 namespace gr {
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                  double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
-                 int* status_out, cudaStream_t st);
+                 int* status_out, FusedArgs fa, cudaStream_t st);
 int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                 double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                cudaStream_t st);
+                FusedArgs fa, cudaStream_t st);
 size_t fullsort_scratch_bytes(int V);
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
                      const char* ws, char* scratch, char* params, int pstride, float* alpha_out, cudaStream_t st);
@@ -23,15 +23,15 @@ void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* bl
 // kernel could not finish, takes the robust kernel.
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                      double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
-                     float* alpha_out, int* status_out, cudaStream_t st)
+                     float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st)
 {
     int rc = force_robust ? 1
                           : launch_fast(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep,
-                                        batch, alpha_out, status_out, st);
+                                        batch, alpha_out, status_out, fa, st);
     if (rc < 0) return rc;
     // rc == 1: no fast variant, the robust kernel does everything; rc == 0: it redoes what the fast one flagged
     return launch_solve(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch,
-                        rc == 0 ? 1 : 0, alpha_out, status_out, st);
+                        rc == 0 ? 1 : 0, alpha_out, status_out, fa, st);
 }
 
 static bool shape_ok(int V, int n, int batch) {
@@ -58,9 +58,9 @@ size_t gr_workspace_bytes(int V, int n, int topk, int batch)
     return s;
 }
 
-int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
-             float temp_draft, int batch, const gr_options* opt, void* params, void* workspace, float* alpha_star,
-             int* status, void* stream)
+static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
+                      float temp_draft, int batch, const gr_options* opt, void* params, void* workspace,
+                      float* alpha_star, int* status, gr::FusedArgs fa, void* stream)
 {
     if (!gr::shape_ok(V, n, batch)) return GR_E_INVALID;
     if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
@@ -93,7 +93,7 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     int rc = gr::launch_solve_any((const char*)workspace, (char*)params, pstride, kcap, V, n, topk,
                                   (double)temp_target, (double)temp_draft, tol, max_iters, qstep, batch, force_robust,
-                                  alpha_star, status, st);
+                                  alpha_star, status, fa, st);
     if (rc != GR_OK) return rc;
     if (full_large) {
         // no rule is solved for this shape, but the optimal acceptance still is (sort + prefix scan)
@@ -103,6 +103,26 @@ int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n
     }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;
+}
+
+int gr_solve(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
+             float temp_draft, int batch, const gr_options* opt, void* params, void* workspace, float* alpha_star,
+             int* status, void* stream)
+{
+    gr::FusedArgs none = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    return solve_impl(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch, opt, params, workspace,
+                      alpha_star, status, none, stream);
+}
+
+int gr_solve_verify(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
+                    float temp_draft, int batch, const gr_options* opt, const int* draft_tokens, const float* uniforms,
+                    void* params, void* workspace, float* alpha_star, int* out_token, unsigned char* out_accepted,
+                    int* status, void* stream)
+{
+    if (batch > 0 && (!draft_tokens || !uniforms || !out_token || !out_accepted)) return GR_E_NULL;
+    gr::FusedArgs fa = {draft_tokens, uniforms, out_token, out_accepted, status};
+    return solve_impl(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch, opt, params, workspace,
+                      alpha_star, status, fa, stream);
 }
 
 int gr_verify(const void* params, const int* draft_tokens, const float* uniforms, int batch, int* out_token,
@@ -138,6 +158,7 @@ const char* gr_strerror(int code)
         case GR_BAD_LOGITS: return "NaN or infinite logit";
         case GR_DRAFT_OUT_OF_SUPPORT: return "drafted token outside the draft support";
         case GR_STALE_PARAMS: return "params block was not written by gr_solve";
+        case GR_PARTIAL_RULE: return "rule solved only for the drafts given to gr_solve_verify";
         case GR_E_INVALID: return "invalid size, temperature or option";
         case GR_E_NULL: return "required pointer is NULL";
         case GR_E_ALIGN: return "pointer is not 16-byte aligned";

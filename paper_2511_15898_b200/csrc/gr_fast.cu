@@ -1,5 +1,5 @@
 // Dispatch of the fast per-instance solve (kernels in gr_fast.cuh, one translation unit per series length).
-#include "gr_common.cuh"
+#include "gr_verify.cuh"
 
 namespace gr {
 
@@ -7,7 +7,8 @@ constexpr int kFastMaxSupport = 64;   // padded support size of the fast kernels
 
 #define GR_FAST_ARGS                                                                                              \
     const char *ws, char *params, int pstride, int kcap, int V, int n, int topk, double temp_t, double temp_d,   \
-        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, cudaStream_t st
+        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, FusedArgs fa,     \
+        cudaStream_t st
 int launch_fast_n4(GR_FAST_ARGS);
 int launch_fast_n8(GR_FAST_ARGS);
 int launch_fast_n16(GR_FAST_ARGS);
@@ -17,7 +18,7 @@ int launch_fast_n16(GR_FAST_ARGS);
 int launch_fast(GR_FAST_ARGS)
 {
     if (kcap <= 0 || kcap > kFastMaxSupport || n > 16 || n < 2) return 1;
-#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, st
+#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, fa, st
     if (n <= 4) return launch_fast_n4(GR_FAST_PASS);
     if (n <= 8) return launch_fast_n8(GR_FAST_PASS);
     return launch_fast_n16(GR_FAST_PASS);

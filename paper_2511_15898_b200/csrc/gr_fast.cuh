@@ -22,6 +22,7 @@
 //     of the other drafted tokens).
 #pragma once
 #include "gr_prep.cuh"
+#include "gr_verify.cuh"
 
 namespace gr {
 
@@ -762,9 +763,11 @@ template <int NT, int TPL>
 __global__ void __launch_bounds__(kFT, kFCtas)
 fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
                   double temp_t, double temp_d, double tol, int max_iters, double qstep,
-                  float* __restrict__ alpha_out, int* __restrict__ status_out)
+                  float* __restrict__ alpha_out, int* __restrict__ status_out, FusedArgs fa)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int s_sel;
+    const bool fused = fa.draft != nullptr;
     const int tid = threadIdx.x;
     const long long b = blockIdx.x;
     char* pb = params + (size_t)b * pstride;
@@ -772,6 +775,10 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     const WsView wv = view_ws(ws, b);
     if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
         if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
+        if (fused) {
+            __syncthreads();
+            fused_draw(fa, pv.h, b, n, smem_raw);
+        }
         return;
     }
     const int KP = kcap;
@@ -798,7 +805,11 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     int status = GR_OK, iters_total = 0;
     double gnorm_total = 0.0;
     if (tid < k) pv.w[tid] = 1.0;
-    if (jstar > 0) {
+    // with the drafted tuple at hand only the system it selects is solved
+    const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
+    bool skipped = false;
+    if (jstar > 0 && sel >= 0) skipped = true;
+    if (jstar > 0 && sel < 0) {
         double gn; int it;
         const int st = fast_system<NT, TPL>(sm, jstar, n, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
         if (st != GR_OK) status = kNeedFallback;
@@ -812,7 +823,8 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
         const int bk = sm.blk[lo];
         while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
         const int m = hi - lo + 1;
-        if (m >= 2) {
+        if (m >= 2 && sel != -2 && sel != bk) skipped = true;
+        if (m >= 2 && (sel == -2 || sel == bk)) {
             double gn; int it;
             const int st = fast_system<NT, TPL>(sm, m, n, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep,
                                                 &gn, &it);
@@ -823,13 +835,18 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
         }
         lo = hi + 1;
     }
+    if (status == GR_OK && skipped) status = GR_PARTIAL_RULE;
     write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
+    if (fused && status != kNeedFallback) {
+        __syncthreads();                       // the rule this CTA wrote is visible to its first warp
+        fused_draw(fa, pv.h, b, n, smem_raw + L.uni * 8);
+    }
 }
 
 template <int NT, int TPL>
 int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                          double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out,
-                         int* status_out, cudaStream_t st)
+                         int* status_out, FusedArgs fa, cudaStream_t st)
 {
     const int smem = fast_smem_bytes(kcap, NT);
     static bool configured = false;
@@ -844,15 +861,16 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
         configured = true;
     }
     fast_solve_kernel<NT, TPL><<<batch, kFT, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
-                                                         max_iters, qstep, alpha_out, status_out);
+                                                         max_iters, qstep, alpha_out, status_out, fa);
     return GR_OK;
 }
 
 // One translation unit per series length instantiates its kernels (they compile in parallel).
 #define GR_FAST_ARGS                                                                                              \
     const char *ws, char *params, int pstride, int kcap, int V, int n, int topk, double temp_t, double temp_d,   \
-        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, cudaStream_t st
-#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, st
+        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, FusedArgs fa,     \
+        cudaStream_t st
+#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, fa, st
 #define GR_FAST_INSTANTIATE(NT)                                                                \
     int launch_fast_n##NT(GR_FAST_ARGS) {                                                       \
         return kcap <= 32 ? launch_fast_t<NT, 1>(GR_FAST_PASS) : launch_fast_t<NT, 2>(GR_FAST_PASS); \

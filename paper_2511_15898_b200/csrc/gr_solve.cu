@@ -17,6 +17,7 @@
 // transition at t ~ 1/w_j on a logarithmic scale and closes the lower tail
 // doubly exponentially.  Newton's method on alpha uses the exact Hessian above.
 #include "gr_prep.cuh"
+#include "gr_verify.cuh"
 
 namespace gr {
 
@@ -444,9 +445,11 @@ __device__ int solve_system(const Sm& sm, int m, const double* d, const double* 
 __global__ void __launch_bounds__(kSolveThreads)
 solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
              double temp_t, double temp_d, double tol, int max_iters, double qstep, int Qt, int only_flagged,
-             float* __restrict__ alpha_out, int* __restrict__ status_out)
+             float* __restrict__ alpha_out, int* __restrict__ status_out, FusedArgs fa)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ int s_sel;
+    const bool fused = fa.draft != nullptr;
     const int tid = threadIdx.x;
     const long long b = blockIdx.x;
     char* pb = params + (size_t)b * pstride;
@@ -457,6 +460,10 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
         // no rule: whole-vocabulary support beyond the capacity, or unusable logits
         if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
+        if (fused) {
+            __syncthreads();
+            fused_draw(fa, pv.h, b, n, smem_raw);
+        }
         return;
     }
 
@@ -486,7 +493,11 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     int status = GR_OK, iters_total = 0;
     double gnorm_total = 0.0;
     if (tid < k) pv.w[tid] = 1.0;
-    if (jstar > 0) {
+    // with the drafted tuple at hand only the system it selects is solved
+    const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
+    bool skipped = false;
+    if (jstar > 0 && sel >= 0) skipped = true;
+    if (jstar > 0 && sel < 0) {
         double gn; int it;
         int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
         if (st != GR_OK) status = GR_NOT_CONVERGED;
@@ -501,7 +512,8 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
             const int bk = sm.blk[lo];
             while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
             const int m = hi - lo + 1;
-            if (m >= 2) {
+            if (m >= 2 && sel != -2 && sel != bk) skipped = true;
+            if (m >= 2 && (sel == -2 || sel == bk)) {
                 double gn; int it;
                 int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it);
                 if (st != GR_OK) status = GR_NOT_CONVERGED;
@@ -513,12 +525,17 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
         }
     }
 
+    if (status == GR_OK && skipped) status = GR_PARTIAL_RULE;
     write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
+    if (fused) {
+        __syncthreads();                       // the rule this CTA wrote is visible to its first warp
+        fused_draw(fa, pv.h, b, n, smem_raw);
+    }
 }
 
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                  double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
-                 int* status_out, cudaStream_t st)
+                 int* status_out, FusedArgs fa, cudaStream_t st)
 {
     int Qt = 1, smem = 0;
     if (kcap > 0) {
@@ -528,6 +545,7 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
         smem = solve_smem_bytes(kcap, n, Qt);
         if (smem > 220 * 1024) return GR_E_TOO_LARGE;
     }
+    if (fa.draft && smem < kVerifyScratchBytes) smem = kVerifyScratchBytes;    // the draw's scratch
     static int configured = 0;
     if (configured < smem) {
         if (cudaFuncSetAttribute(solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
@@ -535,7 +553,7 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
         configured = 220 * 1024;
     }
     solve_kernel<<<batch, kSolveThreads, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
-                                                     max_iters, qstep, Qt, only_flagged, alpha_out, status_out);
+                                                     max_iters, qstep, Qt, only_flagged, alpha_out, status_out, fa);
     return GR_OK;
 }
 

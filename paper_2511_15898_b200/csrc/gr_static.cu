@@ -3,14 +3,14 @@
 // The scratch that gr_solve takes as its `workspace` argument lives here in a
 // file-scope device array instead, so the caller passes inputs and outputs only.
 #include <math.h>
-#include "gr_common.cuh"
+#include "gr_verify.cuh"
 
 namespace gr {
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                      double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
-                     float* alpha_out, int* status_out, cudaStream_t st);
+                     float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st);
 
 constexpr int kStaticBytes = GR_STATIC_MAX_BATCH * (int)(sizeof(WsHeader) + kMaxSupport * 12);
 
@@ -77,7 +77,7 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     const int rc = gr::launch_solve_any(ws, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
                                         (double)temp_draft, tol, max_iters, qstep, batch, force_robust, alpha_star,
-                                        status, st);
+                                        status, gr::FusedArgs{nullptr, nullptr, nullptr, nullptr, nullptr}, st);
     if (rc != GR_OK) return rc;
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;
