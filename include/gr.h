@@ -75,7 +75,7 @@ extern "C" {
  *              the streaming kernel and the solve kernel, so that a caller can
  *              time the two separately; NULL records nothing.      default NULL
  *   force_robust  non-zero sends every shape to the general (slower) solve kernel;
- *              by default supports of at most 64 tokens with n <= 16 take a faster
+ *              by default supports of at most 128 tokens with n <= 16 take a faster
  *              kernel that computes the same rule.                  default 0
  */
 typedef struct gr_options {

@@ -19,7 +19,7 @@ void launch_verify(const char* params, const int* draft, const float* uni, int b
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
                       double* flow, double* header, cudaStream_t st);
 
-// The fast kernel covers supports up to 64 tokens with n <= 16; everything else, and any instance the fast
+// The fast kernel covers supports up to 128 tokens with n <= 16; everything else, and any instance the fast
 // kernel could not finish, takes the robust kernel.
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
                      double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,

@@ -24,18 +24,27 @@
 #include "gr_prep.cuh"
 #include "gr_verify.cuh"
 
-namespace gr {
+// The translation unit that includes this file chooses the padded support size: 64 (96-thread CTAs, four per
+// SM) or 128 (128-thread CTAs, one per SM), and a namespace of its own for the instantiation.
+#ifndef GR_FAST_MP
+#define GR_FAST_MP 64
+#define GR_FAST_NS fast64
+#endif
 
-constexpr int kFT = 96;               // threads per CTA (at least kMP)
-constexpr int kFCtas = 4;             // CTAs per SM the kernels are compiled for
+namespace gr {
+namespace GR_FAST_NS {
+
+constexpr int kMP = GR_FAST_MP;       // padded support size of these kernels
+constexpr int kRL = kMP / 32;         // rows (or tokens) per lane when a warp covers the whole support
+constexpr int kFT = kMP == 64 ? 96 : 128;   // threads per CTA (at least kMP - 8: one thread per panel row)
+constexpr int kFCtas = kMP == 64 ? 4 : 1;   // CTAs per SM the kernels are compiled for
 constexpr int kFW = kFT / 32;         // warps per CTA
-constexpr int kMP = 64;               // padded support size of this kernel
-constexpr int kJC = 6;                // Hessian nodes staged per chunk
+constexpr int kJC = kMP == 64 ? 6 : 4;      // Hessian nodes staged per chunk
 constexpr double kFTEnd = 25.0;       // quadrature range constants, identical to the robust kernel's
 constexpr double kFDrop = 1.0;
 constexpr double kFTail = 3.0;
 constexpr int kFMaxNodes = 128;
-constexpr int kMS = 72;               // row stride of the staged operands (floats): conflict-free MMA fragment loads
+constexpr int kMS = kMP + 8;          // row stride of the staged operands (floats): conflict-free MMA fragment loads
 constexpr int kJS = kMP + 1;          // row stride of the contraction accumulator / Hessian (floats)
 constexpr double kFAlphaClamp = 80.0;
 constexpr double kFStepClamp = 3.0;
@@ -195,15 +204,17 @@ __device__ __forceinline__ void mma_tf32(float& c0, float& c1, float& c2, float&
 
 // One chunk of the Hessian contraction: Jacc[i][l] += sum over the staged rows kk of AS[kk][i] HS[kk][l] for the
 // 16 x 8 tiles that touch the lower triangle, as m16n8k8 tf32 MMAs with fp32 accumulation.  K8 = staged rows,
-// a multiple of 8.  The 20 lower tiles of the 64 x 64 matrix are dealt round-robin to the four warps.
+// a multiple of 8.  The lower tiles are dealt round-robin to the warps.
 template <bool kSplit>
 __device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gid = lane >> 2, tig = lane & 3;
-    for (int t = warp; t < 20; t += kFW) {
-        const int mi = t >= 12 ? 3 : (t >= 6 ? 2 : (t >= 2 ? 1 : 0));
-        const int ni = t - (mi == 3 ? 12 : (mi == 2 ? 6 : (mi == 1 ? 2 : 0)));
+    // tile (mi, ni), ni <= 2 mi + 1, has the running number mi (mi + 1) + ni
+    for (int t = warp; t < (kMP / 16) * (kMP / 16 + 1); t += kFW) {
+        int mi = 0;
+        while ((mi + 1) * (mi + 2) <= t) mi++;
+        const int ni = t - mi * (mi + 1);
         const int i0 = 16 * mi, l0 = 8 * ni;
         if (i0 >= m || l0 >= m) continue;
         float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
@@ -452,7 +463,7 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
     float* dg = yf + kMP;                              // [kMP] diagonal of the factor
     const float addf = (float)add;
     for (int e = tid; e < m * kMP; e += kFT) {
-        const int i = e >> 6, l = e & (kMP - 1);
+        const int i = e / kMP, l = e & (kMP - 1);
         if (l < i) Jm[i * kJS + l] = addf - Jm[i * kJS + l];
     }
     if (tid < m) {
@@ -575,25 +586,40 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
         return;
     }
     // backward substitution L^T x = y on warp 0, column-oriented with the right-hand side in registers (lane l holds
-    // entries l and l + 32): unknown e is finished by its owner, broadcast, and taken out of the entries above it.
+    // entries l, l + 32, ...): unknown e is finished by its owner, broadcast, and taken out of the entries above it.
     // One multiply, one shuffle and one FMA per unknown on the critical path; row e of L is fetched one step ahead.
     if (tid < 32) {
         const int lane = tid;
-        float y0 = lane < m ? yf[lane] : 0.f, y1 = lane + 32 < m ? yf[lane + 32] : 0.f;
-        const float r0 = lane < m ? 1.f / dg[lane] : 0.f, r1 = lane + 32 < m ? 1.f / dg[lane + 32] : 0.f;
-        float a0n = Jm[(m - 1) * kJS + lane], a1n = Jm[(m - 1) * kJS + lane + 32];
-        for (int e = m - 1; e >= 0; e--) {
-            const float a0 = a0n, a1 = a1n;
-            if (e > 0) { a0n = Jm[(e - 1) * kJS + lane]; a1n = Jm[(e - 1) * kJS + lane + 32]; }
-            const float xe = __shfl_sync(0xffffffffu, (e & 32) ? y1 * r1 : y0 * r0, e & 31);
-            if (lane == (e & 31)) {
-                if (e & 32) y1 = xe; else y0 = xe;
-            }
-            if (lane < e) y0 = fmaf(-a0, xe, y0);
-            if (lane + 32 < e) y1 = fmaf(-a1, xe, y1);
+        float y[kRL], rd[kRL], an[kRL];
+#pragma unroll
+        for (int u = 0; u < kRL; u++) {
+            const int l = lane + 32 * u;
+            y[u] = l < m ? yf[l] : 0.f;
+            rd[u] = l < m ? 1.f / dg[l] : 0.f;
+            an[u] = Jm[(m - 1) * kJS + l];
         }
-        if (lane < m) yf[lane] = y0;
-        if (lane + 32 < m) yf[lane + 32] = y1;
+        for (int e = m - 1; e >= 0; e--) {
+            float a[kRL];
+#pragma unroll
+            for (int u = 0; u < kRL; u++) a[u] = an[u];
+            if (e > 0) {
+#pragma unroll
+                for (int u = 0; u < kRL; u++) an[u] = Jm[(e - 1) * kJS + lane + 32 * u];
+            }
+            float xv = 0.f;
+#pragma unroll
+            for (int u = 0; u < kRL; u++) xv = (e >> 5) == u ? y[u] * rd[u] : xv;
+            const float xe = __shfl_sync(0xffffffffu, xv, e & 31);
+#pragma unroll
+            for (int u = 0; u < kRL; u++) {
+                const int l = lane + 32 * u;
+                if (l == e) y[u] = xe;
+                else if (l < e) y[u] = fmaf(-a[u], xe, y[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kRL; u++)
+            if (lane + 32 * u < m) yf[lane + 32 * u] = y[u];
     }
     __syncthreads();
     if (tid < m) sm.delta[tid] = (double)yf[tid];
@@ -643,35 +669,40 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     __syncthreads();
     float* part = sm.AS;                              // [kFW][kMP] partial sums (the staging area is idle here)
     for (int sweep = 0; sweep < kFSweeps; sweep++) {
-        // lane = row (and row + 32), warp = a contiguous share of the columns: no shuffles, four independent sums
+        // lane = rows lane, lane + 32, ...; warp = a contiguous share of the columns: no shuffles, independent sums
         {
             const int chunk = (m + kFW - 1) / kFW;
             const int jlo = warp * chunk, jhi = min(m, jlo + chunk);
-            const int r0 = lane, r1 = lane + 32;
-            const bool on0 = r0 < m, on1 = r1 < m;
-            const float A0 = on0 ? (float)sm.g[r0] : 1.f, c0 = on0 ? (float)sm.g2[r0] : 0.f;
-            const float A1 = on1 ? (float)sm.g[r1] : 1.f, c1 = on1 ? (float)sm.g2[r1] : 0.f;
-            const float* row0 = sm.Jacc + (on0 ? r0 : 0) * kJS;
-            const float* row1 = sm.Jacc + (on1 ? r1 : 0) * kJS;
-            float s0a = 0.f, s0b = 0.f, s1a = 0.f, s1b = 0.f;
+            float Ar[kRL], cr[kRL], sa[kRL], sb[kRL];
+            const float* row[kRL];
+#pragma unroll
+            for (int u = 0; u < kRL; u++) {
+                const int r = lane + 32 * u;
+                const bool on = r < m;
+                Ar[u] = on ? (float)sm.g[r] : 1.f; cr[u] = on ? (float)sm.g2[r] : 0.f;
+                row[u] = sm.Jacc + (on ? r : 0) * kJS;
+                sa[u] = 0.f; sb[u] = 0.f;
+            }
             int j = jlo;
             for (; j + 1 < jhi; j += 2) {
                 const float wa = (float)sm.w[j], wb = (float)sm.w[j + 1];
-                const float p0a = fminf(row0[j] * c0, 1.f), p0b = fminf(row0[j + 1] * c0, 1.f);
-                const float p1a = fminf(row1[j] * c1, 1.f), p1b = fminf(row1[j + 1] * c1, 1.f);
-                s0a += __fdividef(A0 * p0a * wa, A0 + wa * (1.f - p0a));
-                s0b += __fdividef(A0 * p0b * wb, A0 + wb * (1.f - p0b));
-                s1a += __fdividef(A1 * p1a * wa, A1 + wa * (1.f - p1a));
-                s1b += __fdividef(A1 * p1b * wb, A1 + wb * (1.f - p1b));
+#pragma unroll
+                for (int u = 0; u < kRL; u++) {
+                    const float pa = fminf(row[u][j] * cr[u], 1.f), pb = fminf(row[u][j + 1] * cr[u], 1.f);
+                    sa[u] += __fdividef(Ar[u] * pa * wa, Ar[u] + wa * (1.f - pa));
+                    sb[u] += __fdividef(Ar[u] * pb * wb, Ar[u] + wb * (1.f - pb));
+                }
             }
             if (j < jhi) {
                 const float wa = (float)sm.w[j];
-                const float p0a = fminf(row0[j] * c0, 1.f), p1a = fminf(row1[j] * c1, 1.f);
-                s0a += __fdividef(A0 * p0a * wa, A0 + wa * (1.f - p0a));
-                s1a += __fdividef(A1 * p1a * wa, A1 + wa * (1.f - p1a));
+#pragma unroll
+                for (int u = 0; u < kRL; u++) {
+                    const float pa = fminf(row[u][j] * cr[u], 1.f);
+                    sa[u] += __fdividef(Ar[u] * pa * wa, Ar[u] + wa * (1.f - pa));
+                }
             }
-            part[warp * kMP + r0] = s0a + s0b;
-            part[warp * kMP + r1] = s1a + s1b;
+#pragma unroll
+            for (int u = 0; u < kRL; u++) part[warp * kMP + lane + 32 * u] = sa[u] + sb[u];
         }
         __syncthreads();
         double Si = 0.0;
@@ -852,7 +883,7 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 96 * 1024) != cudaSuccess)
+                                 kMP == 64 ? 96 * 1024 : 200 * 1024) != cudaSuccess)
             return GR_E_LAUNCH;
         // the CTAs are small: ask for the largest shared-memory carve-out so that kFCtas of them fit on an SM
         if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -873,7 +904,9 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
 #define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, fa, st
 #define GR_FAST_INSTANTIATE(NT)                                                                \
     int launch_fast_n##NT(GR_FAST_ARGS) {                                                       \
-        return kcap <= 32 ? launch_fast_t<NT, 1>(GR_FAST_PASS) : launch_fast_t<NT, 2>(GR_FAST_PASS); \
+        return kcap <= 32 * (kRL - 1) ? launch_fast_t<NT, kRL - 1>(GR_FAST_PASS)                    \
+                                      : launch_fast_t<NT, kRL>(GR_FAST_PASS);                       \
     }
 
+}  // namespace GR_FAST_NS
 }  // namespace gr
