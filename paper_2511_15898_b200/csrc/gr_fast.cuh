@@ -1,13 +1,13 @@
-// Fast per-instance solve for supports up to 64 tokens and n <= 16 (one 128-thread CTA per
-// instance, several CTAs per SM).
+// Fast per-instance solve for supports up to 128 tokens and n <= 16: one CTA per instance, 96 threads and four
+// CTAs per SM for supports up to 64, 128 threads and one CTA per SM above.
 //
 // Same mathematics as the robust kernel (gr_solve.cu): the gradient of the convex functions
 // of the inner system / of an outer block (Thm "Inner Convex Solver", Thm "Outer Convex Solver")
 // is the one-dimensional integral
 //   g_i = w_i int e^{-t slack} x_i(t) n! [lambda^n] P(lambda; t) h_i(lambda; t) dt,
 // and Newton's method on alpha = log w uses its exact Hessian.  Organised for throughput:
-//   - one warp per quadrature node, one lane per token (two tokens per lane above 32): every
-//     power series lives in registers;
+//   - one warp per quadrature node, one lane per token (up to four tokens per lane on the larger supports):
+//     every power series lives in registers;
 //   - the product P = e^{lambda h} prod_j f_j over the tokens is not multiplied out:
 //     d/dlambda log f_j = x_j d_j (1 + (1 - x_j) h_j), so the log-derivative S of P is a SUM over
 //     tokens (a warp reduction) and P follows from P' = S P.  In fp64 this is accurate to
@@ -19,7 +19,7 @@
 //     taken on every second node (trapezoid step doubled) and accumulated in fp32 from operands
 //     staged in shared memory; the gradient itself stays fp64 on every node;
 //   - the iteration starts from a mean-field point (each token against the expected weight
-//     of the other drafted tokens).
+//     of the other drafted tokens, with a bound on what a single huge competitor can add).
 #pragma once
 #include "gr_prep.cuh"
 #include "gr_verify.cuh"
