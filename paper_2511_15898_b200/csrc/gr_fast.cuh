@@ -588,7 +588,26 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
     // backward substitution L^T x = y on warp 0, column-oriented with the right-hand side in registers (lane l holds
     // entries l, l + 32, ...): unknown e is finished by its owner, broadcast, and taken out of the entries above it.
     // One multiply, one shuffle and one FMA per unknown on the critical path; row e of L is fetched one step ahead.
-    if (tid < 32) {
+    if (tid < 32 && kRL == 2) {
+        // (two entries per lane, written out: the general form below compiles to slower code for them)
+        const int lane = tid;
+        float y0 = lane < m ? yf[lane] : 0.f, y1 = lane + 32 < m ? yf[lane + 32] : 0.f;
+        const float r0 = lane < m ? 1.f / dg[lane] : 0.f, r1 = lane + 32 < m ? 1.f / dg[lane + 32] : 0.f;
+        float a0n = Jm[(m - 1) * kJS + lane], a1n = Jm[(m - 1) * kJS + lane + 32];
+        for (int e = m - 1; e >= 0; e--) {
+            const float a0 = a0n, a1 = a1n;
+            if (e > 0) { a0n = Jm[(e - 1) * kJS + lane]; a1n = Jm[(e - 1) * kJS + lane + 32]; }
+            const float xe = __shfl_sync(0xffffffffu, (e & 32) ? y1 * r1 : y0 * r0, e & 31);
+            if (lane == (e & 31)) {
+                if (e & 32) y1 = xe; else y0 = xe;
+            }
+            if (lane < e) y0 = fmaf(-a0, xe, y0);
+            if (lane + 32 < e) y1 = fmaf(-a1, xe, y1);
+        }
+        if (lane < m) yf[lane] = y0;
+        if (lane + 32 < m) yf[lane + 32] = y1;
+    }
+    if (tid < 32 && kRL != 2) {
         const int lane = tid;
         float y[kRL], rd[kRL], an[kRL];
 #pragma unroll

@@ -107,6 +107,14 @@ __device__ float refine_tau(float lmax, int need) {
     return fkey_inv(res);
 }
 
+// one lane's element
+__device__ __forceinline__ void push_lane(const CandList& cl, float val, int id, float tau) {
+    if (val >= tau) {
+        const int slot = atomicAdd(cl.cnt, 1);
+        if (slot < kCandCap) { cl.v[slot] = val; cl.id[slot] = id; }
+    }
+}
+
 // Exact selection of the ksel largest composite keys of the draft row by eight 8-bit
 // radix passes over the row (slow path, taken only when the candidate list overflowed).
 template <typename T>
@@ -213,6 +221,10 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
             tsum += x; dsum += v; lmax = fmaxf(lmax, v);
             if (kFull) osm_update<1>(dm, dsum_e, &v, sc_d);
         }
+        // Batches of U vector steps.  A candidate (draft logit >= tau) is appended by its own lane, without any warp
+        // vote: about one element in four hundred is one, and the list's order does not matter (the exact selection
+        // sorts it).  The CTA's very first batch has no threshold yet: it derives one afterwards and reads its
+        // draft vectors once more (from cache) to test them.
 #pragma unroll 1
         for (int nb = 0; nb < NB; nb++) {
             typename VT::Vec qv[U], pv[U];
@@ -227,41 +239,38 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
                     pv[u] = __ldcs(reinterpret_cast<const typename VT::Vec*>(prow + idx[u]));
                 }
             }
-            float dv[U][N];
-            float tau = use_tau ? *((volatile float*)&s_tau) : -INFINITY;
-            const bool sample = use_tau && (r == 0) && (nb == 0);   // first batch: threshold not known yet
+            const bool sample = use_tau && (r == 0) && (nb == 0);
+            // (+inf on the first batch: nothing passes the in-loop test)
+            const float tau = sample ? INFINITY : (use_tau ? *((volatile float*)&s_tau) : -INFINITY);
 #pragma unroll
             for (int u = 0; u < U; u++) {
-                float tv[N];
                 if (ok[u]) {
+                    float tv[N], dv[N];
                     VT::unpack(qv[u], tv);
-                    VT::unpack(pv[u], dv[u]);
+                    VT::unpack(pv[u], dv);
                     osm_update<N>(cm, cs, tv, sc_t);
-                    if (kFull) osm_update<N>(dm, dsum_e, dv[u], sc_d);
-                    float vm = dv[u][0];
+                    if (kFull) osm_update<N>(dm, dsum_e, dv, sc_d);
+                    float vm = dv[0];
 #pragma unroll
-                    for (int i = 0; i < N; i++) { tsum += tv[i]; dsum += dv[u][i]; vm = fmaxf(vm, dv[u][i]); }
+                    for (int i = 0; i < N; i++) { tsum += tv[i]; dsum += dv[i]; vm = fmaxf(vm, dv[i]); }
                     lmax = fmaxf(lmax, vm);
-                } else {
+                    if (!kFull && vm >= tau) {
 #pragma unroll
-                    for (int i = 0; i < N; i++) dv[u][i] = -INFINITY;
+                        for (int i = 0; i < N; i++) push_lane(cl, dv[i], idx[u] + i, tau);
+                    }
                 }
             }
-            if (!kFull) {
-                if (sample) {
-                    float t0 = refine_tau(lmax, ksel);      // contains CTA-wide barriers; every warp gets here
-                    if (tid == 0) s_tau = fmaxf(s_tau, t0);
-                    __syncthreads();
-                    tau = *((volatile float*)&s_tau);
-                }
-#pragma unroll
+            if (!kFull && sample) {
+                float t0 = refine_tau(lmax, ksel);      // contains CTA-wide barriers; every warp gets here
+                if (tid == 0) s_tau = fmaxf(s_tau, t0);
+                __syncthreads();
+                const float tau1 = *((volatile float*)&s_tau);
                 for (int u = 0; u < U; u++) {
-                    float vm = dv[u][0];
+                    if (ok[u]) {
+                        float dv[N];
+                        VT::unpack(*reinterpret_cast<const typename VT::Vec*>(prow + idx[u]), dv);
 #pragma unroll
-                    for (int i = 1; i < N; i++) vm = fmaxf(vm, dv[u][i]);
-                    if (__any_sync(0xffffffffu, ok[u] && vm >= tau)) {
-#pragma unroll
-                        for (int i = 0; i < N; i++) push_one(cl, dv[u][i], idx[u] + i, ok[u], tau, lane);
+                        for (int i = 0; i < N; i++) push_lane(cl, dv[i], idx[u] + i, tau1);
                     }
                 }
             }
