@@ -205,6 +205,24 @@ int gr_solve_verify(const void* q_logits, const void* p_logits, int dtype, int V
                     void* stream);
 
 /*
+ * gr_alpha_star -- the optimal acceptance alpha* = 1 + min_H psi(H) alone (Eq. "subset-select"), for up to
+ * GR_MAX_ALPHA_N draft counts at once: one pass over the logits (the same streaming kernel as gr_solve) and a
+ * prefix scan along the ratio order, which all the draft counts share.  No rule is solved and no params block
+ * is written; this is what an acceptance-versus-(n, k) sweep needs.
+ *   n_list      HOST array of n_count draft counts, each in 1..GR_MAX_DRAFTS.
+ *   workspace   scratch of gr_workspace_bytes(V, 1, topk, batch) bytes, 16-byte aligned.
+ *   alpha_star  out [batch, n_count] float, row-major; NaN where status is not GR_OK.
+ *   status      out [batch]: GR_OK or GR_BAD_LOGITS.
+ * Supports as for the rule: top-k up to GR_MAX_SUPPORT, or the whole vocabulary when V <= GR_MAX_SUPPORT;
+ * an untruncated draft on a larger vocabulary returns GR_E_TOO_LARGE (gr_solve still gives its alpha*).
+ * Other return values as gr_solve.
+ */
+#define GR_MAX_ALPHA_N 8
+int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, const int* n_list, int n_count,
+                  int topk, float temp_target, float temp_draft, int batch, void* workspace,
+                  float* alpha_star, int* status, void* stream);
+
+/*
  * gr_read_rule -- copies the rule of every instance out of `params` into plain
  * arrays (for inspection and tests); all outputs are optional (NULL skips).
  * Per-support arrays have `kcap` entries per instance and are filled in ratio

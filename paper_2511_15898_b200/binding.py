@@ -65,6 +65,9 @@ def load_library():
     lib.gr_solve_verify.restype = C.c_int
     lib.gr_solve_verify.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int,
                                     C.POINTER(Options), ip, fp, vp, vp, fp, ip, vp, ip, vp]
+    lib.gr_alpha_star.restype = C.c_int
+    lib.gr_alpha_star.argtypes = [vp, vp, C.c_int, C.c_int, ip, C.c_int, C.c_int, C.c_float, C.c_float, C.c_int, vp,
+                                  fp, ip, vp]
     lib.gr_verify.restype = C.c_int
     lib.gr_verify.argtypes = [vp, ip, fp, C.c_int, ip, vp, ip, vp]
     lib.gr_read_rule.restype = C.c_int
@@ -114,6 +117,13 @@ def gr_solve_verify(q_logits: int, p_logits: int, dtype: int, V: int, n: int, to
     return int(load_library().gr_solve_verify(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch,
                                               C.byref(opt) if opt is not None else None, draft_tokens, uniforms,
                                               params, workspace, alpha_star, out_token, out_accepted, status, stream))
+
+
+def gr_alpha_star(q_logits: int, p_logits: int, dtype: int, V: int, n_list, topk: int, temp_target: float,
+                  temp_draft: float, batch: int, workspace: int, alpha_star: int, status: int, stream: int) -> int:
+    ns = (C.c_int * len(n_list))(*[int(x) for x in n_list])
+    return int(load_library().gr_alpha_star(q_logits, p_logits, dtype, V, ns, len(n_list), topk, temp_target,
+                                            temp_draft, batch, workspace, alpha_star, status, stream))
 
 
 def gr_verify(params: int, draft_tokens: int, uniforms: int, batch: int, out_token: int, out_accepted: int,
@@ -216,6 +226,26 @@ def verify(solved: Solved, draft_tokens: torch.Tensor, uniforms: torch.Tensor,
                    out.accepted.data_ptr(), out.status.data_ptr(), _stream())
     _check(rc, "gr_verify")
     return out
+
+
+def alpha_star(q_logits: torch.Tensor, p_logits: torch.Tensor, n_list, topk: int, temp_target: float = 1.0,
+               temp_draft: float = 1.0) -> Tuple[torch.Tensor, torch.Tensor]:
+    """gr_alpha_star on torch CUDA tensors: ([B, len(n_list)] float32 optimal acceptances, [B] int32 status)."""
+    _need_cuda(q_logits, p_logits)
+    if q_logits.shape != p_logits.shape or q_logits.dim() != 2 or q_logits.dtype != p_logits.dtype:
+        raise GrError("q_logits and p_logits must be [B, V] tensors of one dtype")
+    B, V = q_logits.shape
+    dev = q_logits.device
+    wbytes = gr_workspace_bytes(V, 1, topk, B)
+    if wbytes == 0:
+        raise GrError("invalid shape")
+    ws = torch.empty(wbytes, dtype=torch.uint8, device=dev)
+    out = torch.empty((B, len(n_list)), dtype=torch.float32, device=dev)
+    st = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = gr_alpha_star(q_logits.data_ptr(), p_logits.data_ptr(), _dtype_code(q_logits), V, n_list, topk, temp_target,
+                       temp_draft, B, ws.data_ptr(), out.data_ptr(), st.data_ptr(), _stream())
+    _check(rc, "gr_alpha_star")
+    return out, st
 
 
 def solve_verify(q_logits: torch.Tensor, p_logits: torch.Tensor, draft_tokens: torch.Tensor, uniforms: torch.Tensor,

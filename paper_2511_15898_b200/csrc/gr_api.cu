@@ -14,6 +14,8 @@ int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int 
 size_t fullsort_scratch_bytes(int V);
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
                      const char* ws, char* scratch, char* params, int pstride, float* alpha_out, cudaStream_t st);
+void launch_alpha(const char* ws, int V, int topk, double temp_t, double temp_d, const int* n_list, int n_count,
+                  int batch, float* alpha_out, int* status_out, cudaStream_t st);
 void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
                    unsigned char* out_acc, int* status, cudaStream_t st);
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
@@ -123,6 +125,33 @@ int gr_solve_verify(const void* q_logits, const void* p_logits, int dtype, int V
     gr::FusedArgs fa = {draft_tokens, uniforms, out_token, out_accepted, status};
     return solve_impl(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch, opt, params, workspace,
                       alpha_star, status, fa, stream);
+}
+
+int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, const int* n_list, int n_count,
+                  int topk, float temp_target, float temp_draft, int batch, void* workspace, float* alpha_star,
+                  int* status, void* stream)
+{
+    if (!gr::shape_ok(V, 1, batch)) return GR_E_INVALID;
+    if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
+    if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
+        return GR_E_INVALID;
+    if (!n_list) return GR_E_NULL;
+    if (n_count < 1 || n_count > GR_MAX_ALPHA_N) return GR_E_INVALID;
+    for (int i = 0; i < n_count; i++)
+        if (n_list[i] < 1 || n_list[i] > gr::kMaxDrafts) return GR_E_INVALID;
+    if (batch == 0) return GR_OK;
+    if (!q_logits || !p_logits || !workspace || !alpha_star || !status) return GR_E_NULL;
+    if (((uintptr_t)q_logits & 15) || ((uintptr_t)p_logits & 15) || ((uintptr_t)workspace & 15)) return GR_E_ALIGN;
+    const int kfull = (topk <= 0 || topk >= V) ? V : topk;
+    const int kcap = gr::kcap_of(V, topk);
+    if (kcap == 0) return GR_E_TOO_LARGE;
+    cudaStream_t st = (cudaStream_t)stream;
+    gr::launch_scan(q_logits, p_logits, dtype, V, kfull, false, (double)temp_target, (double)temp_draft, batch,
+                    (char*)workspace, nullptr, 0, kcap, st);
+    gr::launch_alpha((const char*)workspace, V, topk, (double)temp_target, (double)temp_draft, n_list, n_count, batch,
+                     alpha_star, status, st);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    return GR_OK;
 }
 
 int gr_verify(const void* params, const int* draft_tokens, const float* uniforms, int batch, int* out_token,

@@ -379,15 +379,19 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
     }
 
     // ---- outputs: workspace header, chunk table and the header fields owned by this kernel
-    char* pb = params + (size_t)b * pstride;
-    ParamView pv = view_params(pb, kcap);
-    for (int c = tid; c < nch; c += kScanThreads) pv.chunk[c] = s_chunk[c];
+    // (params == nullptr: the caller wants the workspace record only)
     if (tid == 0) {
         WsHeader* wh = reinterpret_cast<WsHeader*>(ws + (size_t)b * ws_stride());
         wh->lse_t = s_lse[0];
         wh->lse_d = s_lse[1];
         wh->count = nsel;
         wh->bad = s_bad;
+    }
+    if (params == nullptr) return;
+    char* pb = params + (size_t)b * pstride;
+    ParamView pv = view_params(pb, kcap);
+    for (int c = tid; c < nch; c += kScanThreads) pv.chunk[c] = s_chunk[c];
+    if (tid == 0) {
         Header* h = pv.h;
         h->magic = 0;            // completed by the solve kernel
         h->V = V; h->nch = nch; h->head = head;
