@@ -58,6 +58,13 @@ def test_config5_bf16_top100():
     _check(P.compare(W.config5(batch=4, device="cuda", rows_per_pass=4)))
 
 
+@pytest.mark.parametrize("n,topk", [(3, 70), (6, 80), (8, 128), (12, 90), (16, 128)])
+def test_supports_of_65_to_128_tokens(n, topk):
+    """The wider variant of the fast kernel: three or four tokens per lane, series length 8 and 16."""
+    wl = W.config3(batch=6, device="cuda", seed=3100 + n, V=20000, n=n, topk=topk)
+    _check(P.compare(wl))
+
+
 def test_ragged_rows_and_unaligned_vocabulary():
     """V not a multiple of the vector width or of the chunk: scalar head / tail paths."""
     for V, n, k in [(1031, 3, 6), (4099, 2, 4), (50257, 4, 5)]:
