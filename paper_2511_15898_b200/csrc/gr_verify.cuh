@@ -94,36 +94,40 @@ __device__ inline int resample_draw(const Header* h, const ParamView& pv, int k,
         nl += __popc(mk);
     }
     __syncwarp();
-    // exact pass: every lane owns a contiguous piece of the chunk
-    const int len = ce - cb;
-    const int per = (len + 31) / 32;
-    const int b0 = cb + lane * per, b1 = min(ce, b0 + per);
-    double mysum = 0.0;
-    for (int i = b0; i < b1; i++) {
-        double res = exp((double)load_logit_dyn(row, dtype, i) / T - lse);
-        for (int s = 0; s < nl; s++) if (l_id[s] == i) res = l_r[s];
-        mysum += res;
-    }
-    const double inc = warp_incl_scan(mysum, lane);
+    // exact pass over the chunk in id order, 32 consecutive ids at a time (one per lane): the first id whose running
+    // total exceeds the threshold; the last id of positive residual when rounding left the threshold above the total
     const double want = before < 0.0 ? 1.0e300 : thr - before;
-    const unsigned hit = __ballot_sync(0xffffffffu, inc > want);
-    const unsigned posl = __ballot_sync(0xffffffffu, mysum > 0.0);
-    int owner = hit ? __ffs(hit) - 1 : (posl ? 31 - __clz(posl) : -1);
-    if (owner < 0) return -1;
-    int token = -1;
-    if (lane == owner) {
-        double acc = inc - mysum;
-        int lastp = -1;
-        for (int i = b0; i < b1; i++) {
-            double res = exp((double)load_logit_dyn(row, dtype, i) / T - lse);
-            for (int s = 0; s < nl; s++) if (l_id[s] == i) res = l_r[s];
-            acc += res;
-            if (res > 0.0) lastp = i;
-            if (acc > want) { token = i; break; }
+    double run2 = 0.0;
+    int token = -1, lastp = -1;
+    constexpr int kRows = 8;                 // rows of 32 ids whose logits are fetched together
+    for (int g0 = cb; g0 < ce && token < 0; g0 += 32 * kRows) {
+        float lg[kRows];
+#pragma unroll
+        for (int q = 0; q < kRows; q++) {
+            const int i = g0 + 32 * q + lane;
+            lg[q] = i < ce ? load_logit_dyn(row, dtype, i) : 0.f;
         }
-        if (token < 0) token = lastp;
+#pragma unroll
+        for (int q = 0; q < kRows; q++) {
+            const int r0 = g0 + 32 * q;
+            if (r0 < ce && token < 0) {
+                const int i = r0 + lane;
+                const bool in = i < ce;
+                double res = 0.0;
+                if (in) {
+                    res = exp((double)lg[q] / T - lse);
+                    for (int s2 = 0; s2 < nl; s2++) if (l_id[s2] == i) res = l_r[s2];
+                }
+                const double inc = warp_incl_scan(res, lane) + run2;
+                const unsigned hit = __ballot_sync(0xffffffffu, in && inc > want);
+                const unsigned posl = __ballot_sync(0xffffffffu, in && res > 0.0);
+                if (posl) lastp = r0 + 31 - __clz(posl);
+                if (hit) token = r0 + __ffs(hit) - 1;
+                run2 = __shfl_sync(0xffffffffu, inc, 31);
+            }
+        }
     }
-    return __shfl_sync(0xffffffffu, token, owner);
+    return token >= 0 ? token : lastp;
 }
 
 
