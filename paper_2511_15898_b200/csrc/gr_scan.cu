@@ -95,11 +95,11 @@ __device__ __forceinline__ void push_one(const CandList& cl, float val, int id, 
     }
 }
 
-// largest tau (to 20 leading key bits) such that at least `need` threads hold a running maximum >= tau
+// largest tau (to 16 leading key bits) such that at least `need` threads hold a running maximum >= tau
 __device__ float refine_tau(float lmax, int need) {
     uint32_t key = fkey(lmax);
     uint32_t res = 0;
-    for (int bit = 31; bit >= 12; bit--) {
+    for (int bit = 31; bit >= 16; bit--) {
         uint32_t t = res | (1u << bit);
         int c = __syncthreads_count(key >= t);
         if (c >= need) res = t;
@@ -278,7 +278,7 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
         // chunk result
         osm_warp_reduce(cm, cs, sc_t);
         if (cvalid && lane == 0) s_chunk[c] = make_float2(cm, cs);
-        if (use_tau && r < 2 && r + 1 < rounds) {
+        if (use_tau && r < 4 && r + 1 < rounds) {
             float t1 = refine_tau(lmax, ksel);
             if (tid == 0) s_tau = fmaxf(s_tau, t1);
             __syncthreads();
