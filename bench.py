@@ -32,7 +32,7 @@ HEADLINE = dict(V=128256, n=8, topk=50, batch=1024, temp_target=0.7, temp_draft=
 BYTES_PER_INSTANCE = HEADLINE["V"] * (4 + 4)       # both fp32 logit rows, read once
 # dram__bytes_read + dram__bytes_write of scan_kernel per instance, from the ncu capture at batch 296
 # (profiles/scan_kernel_config3_batch296.md); traffic is proportional to the rows read
-SCAN_TRAFFIC_PER_INSTANCE = (305.112832e6 + 3.397120e6) / 296
+SCAN_TRAFFIC_PER_INSTANCE = (305.128704e6 + 4.365568e6) / 296
 
 
 def _peaks():
