@@ -476,9 +476,11 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
         // token close to saturation (weight in the thousands) is placed at once, where the plain residual moves
         // its weight by a factor e per step, and a light token gets the multiplicative update log(rhs_i / g_i).
         const double gi = sm.g[tid], g2i = sm.g2[tid], ri = rhs[tid];
-        const double den = gi * fmax(1.0 - ri * g2i / (gi * gi), 1e-3);
-        const double arg = fmax((ri - gi) / den, -1.0 + 1e-12);
-        yv[tid] = (float)((gi - g2i) * log1p(arg));
+        // (a target at or beyond the saturation level this curve predicts says that the curve is off: the plain
+        // residual is used for that token; without this a single token of weight ~1e5 crawled for 40 steps)
+        const double room = 1.0 - ri * g2i / (gi * gi);
+        const double arg = fmax((ri - gi) / (gi * fmax(room, 1e-3)), -1.0 + 1e-12);
+        yv[tid] = (float)(room > 1e-3 ? (gi - g2i) * log1p(arg) : ri - gi);
     }
     __syncthreads();
     bool bad = false;

@@ -65,6 +65,22 @@ def test_supports_of_65_to_128_tokens(n, topk):
     _check(P.compare(wl))
 
 
+def test_low_target_temperature_with_a_saturated_token():
+    """Sharper target (temperature 0.5): acceptance ~0.94 and single tokens that must win nearly every tuple they
+    are in (weights up to ~1e5).  Parity on a slice, and on a larger batch every instance converges in few steps."""
+    base = W.config3(batch=512, device="cuda", seed=77)
+    g = torch.Generator(device="cuda"); g.manual_seed(78)
+    p = base.q_logits + 0.75 * torch.randn(base.q_logits.shape, generator=g, device="cuda")
+    wl = W._finish("config3 at target temperature 0.5", base.V, base.n, base.topk, 0.5, 1.0, base.q_logits, p, g)
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+    rule = G.read_rule(solved)
+    torch.cuda.synchronize()
+    assert solved.status.cpu().tolist() == [G.GR_OK] * wl.batch
+    assert float(rule.w.max()) > 1e4            # the saturated regime is present in this batch
+    assert int(rule.iters.max()) <= 15
+    _check(P.compare(wl.rows(list(range(416, 440)))))      # includes the heaviest instance (428)
+
+
 def test_ragged_rows_and_unaligned_vocabulary():
     """V not a multiple of the vector width or of the chunk: scalar head / tail paths."""
     for V, n, k in [(1031, 3, 6), (4099, 2, 4), (50257, 4, 5)]:
