@@ -73,11 +73,27 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert G.gr_verify(A, A, A, -1, A, A, A, 0) == -1
     assert G.gr_verify(A, A, A, 0, A, A, A, 0) == 0
     assert G.gr_read_rule(0, 1, 8, 0, 0, 0, 0, 0, 0, 0) == -2
+    # the fused entry: gr_solve's checks plus its own pointers
+    def fused(**kw):
+        a = dict(ok); a.update(kw)
+        return G.gr_solve_verify(a["q"], a["p"], a["dtype"], a["V"], a["n"], a["topk"], a["tt"], a["td"], a["batch"],
+                                 None, a.get("draft", A), a.get("uni", A), A, A, A, a.get("tok", A), A, A, 0)
+    assert fused(draft=0) == -2 and fused(uni=0) == -2 and fused(tok=0) == -2
+    assert fused(V=0) == -1 and fused(q=A + 4) == -3 and fused(batch=0) == 0
+    # the acceptance-only entry
+    def alpha(ns, **kw):
+        a = dict(ok); a.update(kw)
+        return G.gr_alpha_star(a["q"], a["p"], a["dtype"], a["V"], ns, a["topk"], a["tt"], a["td"], a["batch"], A, A,
+                               A, 0)
+    assert alpha([]) == -1 and alpha([0]) == -1 and alpha([33]) == -1 and alpha(list(range(1, 10))) == -1
+    assert alpha([2], q=0) == -2 and alpha([2], q=A + 4) == -3 and alpha([2], tt=0.0) == -1
+    assert alpha([2], V=100000, topk=0) == -5   # untruncated draft beyond GR_MAX_SUPPORT
+    assert alpha([2, 4], batch=0) == 0
 
 
 def test_strerror(lib):
     assert G.gr_strerror(0) == "ok"
-    for code in (1, 2, 3, 4, 5, -1, -2, -3, -4, -5):
+    for code in (1, 2, 3, 4, 5, 6, -1, -2, -3, -4, -5):
         assert G.gr_strerror(code) not in ("", "unknown code")
     assert G.gr_strerror(99) == "unknown code"
 
@@ -87,6 +103,10 @@ def test_tensor_front_end_refuses_cpu_tensors(lib):
     q = torch.zeros(2, 16)
     with pytest.raises(G.GrError):
         G.solve(q, q, 2, 0)
+    with pytest.raises(G.GrError):
+        G.alpha_star(q, q, [2], 0)
+    with pytest.raises(G.GrError):
+        G.solve_verify(q, q, torch.zeros(2, 2, dtype=torch.int32), torch.zeros(2, 2), 0)
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
