@@ -12,7 +12,7 @@ LIB = os.path.join(HERE, "libgr_b200.so")
 OBJ = os.path.join(HERE, "_build")
 SOURCES = ["gr_api.cu", "gr_alpha.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_fast_n4.cu", "gr_fast_n8.cu",
            "gr_fast_n16.cu", "gr_fast_w8.cu", "gr_fast_w16.cu", "gr_fullsort.cu", "gr_verify.cu"]
-HEADERS = [os.path.join(CSRC, "gr_common.cuh"), os.path.join(CSRC, "gr_prep.cuh"), os.path.join(CSRC, "gr_fast.cuh"), os.path.join(CSRC, "gr_verify.cuh"),
+HEADERS = [os.path.join(CSRC, "gr_common.cuh"), os.path.join(CSRC, "gr_prep.cuh"), os.path.join(CSRC, "gr_fast.cuh"), os.path.join(CSRC, "gr_verify.cuh"), os.path.join(CSRC, "gr_host.h"),
            os.path.join(ROOT, "include", "gr.h")]
 
 

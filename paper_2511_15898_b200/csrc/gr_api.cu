@@ -1,26 +1,8 @@
 // Host side of the C interface declared in gr.h: argument checks and kernel launches.
 #include <math.h>
-#include "gr_verify.cuh"
+#include "gr_host.h"
 
 namespace gr {
-void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
-                 double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
-int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
-                 int* status_out, FusedArgs fa, cudaStream_t st);
-int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                FusedArgs fa, cudaStream_t st);
-size_t fullsort_scratch_bytes(int V);
-void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
-                     const char* ws, char* scratch, char* params, int pstride, float* alpha_out, cudaStream_t st);
-void launch_alpha(const char* ws, int V, int topk, double temp_t, double temp_d, const int* n_list, int n_count,
-                  int batch, float* alpha_out, int* status_out, cudaStream_t st);
-void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
-                   unsigned char* out_acc, int* status, cudaStream_t st);
-void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
-                      double* flow, double* header, cudaStream_t st);
-
 // The fast kernel covers supports up to 128 tokens with n <= 16; everything else, and any instance the fast
 // kernel could not finish, takes the robust kernel.
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
@@ -38,6 +20,32 @@ int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V,
 
 static bool shape_ok(int V, int n, int batch) {
     return V >= 1 && V <= (1 << 21) && n >= 1 && n <= kMaxDrafts && batch >= 0;
+}
+
+int check_solve_args(const void* q_logits, const void* p_logits, int dtype, int V, int n, int topk, float temp_target,
+                     float temp_draft, int batch, const gr_options* opt, const void* params, const float* alpha_star,
+                     const int* status, SolveSetup* out)
+{
+    if (!shape_ok(V, n, batch)) return GR_E_INVALID;
+    if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
+    if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
+        return GR_E_INVALID;
+    out->tol = 1e-9; out->qstep = 0.4; out->max_iters = 40;
+    out->scan_done = nullptr; out->force_robust = 0;
+    if (opt) {
+        out->scan_done = (cudaEvent_t)opt->scan_done_event;
+        out->force_robust = opt->force_robust;
+        out->tol = opt->tol; out->max_iters = opt->max_iters; out->qstep = opt->quad_step;
+        if (!(out->tol > 0.0) || out->max_iters < 1 || !(out->qstep >= 0.05 && out->qstep <= 2.0)) return GR_E_INVALID;
+    }
+    out->kfull = (topk <= 0 || topk >= V) ? V : topk;
+    out->kcap = kcap_of(V, topk);
+    out->pstride = params_stride(V, topk);
+    if (batch == 0) return GR_OK;
+    if (!q_logits || !p_logits || !params || !alpha_star || !status) return GR_E_NULL;
+    if (((uintptr_t)q_logits & 15) || ((uintptr_t)p_logits & 15) || ((uintptr_t)params & 15)) return GR_E_ALIGN;
+    if (out->kcap == 0 && out->kfull != V) return GR_E_TOO_LARGE;   // a truncated support beyond the capacity
+    return GR_OK;
 }
 }  // namespace gr
 
@@ -64,30 +72,18 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
                       float temp_draft, int batch, const gr_options* opt, void* params, void* workspace,
                       float* alpha_star, int* status, gr::FusedArgs fa, void* stream)
 {
-    if (!gr::shape_ok(V, n, batch)) return GR_E_INVALID;
-    if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
-    if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
-        return GR_E_INVALID;
-    double tol = 1e-9, qstep = 0.4;
-    int max_iters = 40;
-    cudaEvent_t scan_done = nullptr;
-    int force_robust = 0;
-    if (opt) {
-        scan_done = (cudaEvent_t)opt->scan_done_event;
-        force_robust = opt->force_robust;
-        tol = opt->tol; max_iters = opt->max_iters; qstep = opt->quad_step;
-        if (!(tol > 0.0) || max_iters < 1 || !(qstep >= 0.05 && qstep <= 2.0)) return GR_E_INVALID;
-    }
+    gr::SolveSetup su;
+    const int chk = gr::check_solve_args(q_logits, p_logits, dtype, V, n, topk, temp_target, temp_draft, batch, opt,
+                                         params, alpha_star, status, &su);
+    if (chk != GR_OK) return chk;
     if (batch == 0) return GR_OK;
-    if (!q_logits || !p_logits || !params || !workspace || !alpha_star || !status) return GR_E_NULL;
-    if (((uintptr_t)q_logits & 15) || ((uintptr_t)p_logits & 15) || ((uintptr_t)params & 15) ||
-        ((uintptr_t)workspace & 15))
-        return GR_E_ALIGN;
-    const int kfull = (topk <= 0 || topk >= V) ? V : topk;
-    const int kcap = gr::kcap_of(V, topk);
+    if (!workspace) return GR_E_NULL;
+    if ((uintptr_t)workspace & 15) return GR_E_ALIGN;
+    const double tol = su.tol, qstep = su.qstep;
+    const int max_iters = su.max_iters, force_robust = su.force_robust;
+    cudaEvent_t scan_done = su.scan_done;
+    const int kfull = su.kfull, kcap = su.kcap, pstride = su.pstride;
     const bool full_large = kcap == 0;
-    if (full_large && kfull != V) return GR_E_TOO_LARGE;   // a truncated support beyond the capacity
-    const int pstride = gr::params_stride(V, topk);
     cudaStream_t st = (cudaStream_t)stream;
     gr::launch_scan(q_logits, p_logits, dtype, V, kfull, full_large, (double)temp_target, (double)temp_draft, batch,
                     (char*)workspace, (char*)params, pstride, kcap, st);

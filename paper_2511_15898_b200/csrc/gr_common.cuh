@@ -112,7 +112,7 @@ __device__ inline float load_logit_dyn(const void* row, int dtype, int i) {
 
 // order-preserving map float -> uint32 (larger float, larger key)
 __device__ inline uint32_t fkey(float f) {
-    uint32_t u = __float_as_uint(f);
+    uint32_t u = __float_as_uint(f + 0.f);       // (-0 + 0 = +0: the two zeros compare equal, so they get one key)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 __device__ inline float fkey_inv(uint32_t k) {
@@ -124,11 +124,6 @@ __device__ inline unsigned long long ckey(float v, int id) {
     return ((unsigned long long)fkey(v) << 32) | (unsigned long long)(0xffffffffu - (uint32_t)id);
 }
 
-struct SolveArgs {
-    int V, n, topk, batch, dtype;
-    double inv_temp_target_unused;
-    double temp_target, temp_draft;
-    double tol; int max_iters; double quad_step;
-};
+constexpr int kMaxDevices = 64;               // per-device caches of the host code (function attributes, streams)
 
 }  // namespace gr

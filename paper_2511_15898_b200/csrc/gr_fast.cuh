@@ -901,8 +901,11 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
                          int* status_out, FusedArgs fa, cudaStream_t st)
 {
     const int smem = fast_smem_bytes(kcap, NT);
-    static bool configured = false;
-    if (!configured) {
+    // function attributes belong to the device: set once per device
+    static bool configured[kMaxDevices] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return GR_E_LAUNCH; }
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kMP == 64 ? 96 * 1024 : 200 * 1024) != cudaSuccess)
             return GR_E_LAUNCH;
@@ -910,7 +913,7 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
         if (cudaFuncSetAttribute(fast_solve_kernel<NT, TPL>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                  cudaSharedmemCarveoutMaxShared) != cudaSuccess)
             return GR_E_LAUNCH;
-        configured = true;
+        configured[dev] = true;
     }
     fast_solve_kernel<NT, TPL><<<batch, kFT, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
                                                          max_iters, qstep, alpha_out, status_out, fa);

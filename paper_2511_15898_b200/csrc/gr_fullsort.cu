@@ -189,12 +189,16 @@ fullsort_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, i
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
                      const char* ws, char* scratch, char* params, int pstride, float* alpha_out, cudaStream_t st)
 {
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(fullsort_alpha_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes);
-        cudaFuncSetAttribute(fullsort_alpha_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             kFsSmemBytes);
-        configured = true;
+    // function attributes belong to the device: set once per device (a failure shows up as a launch error)
+    static bool configured[kMaxDevices] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) dev = -1;
+    if (dev < 0 || !configured[dev]) {
+        const bool ok = cudaFuncSetAttribute(fullsort_alpha_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kFsSmemBytes) == cudaSuccess &&
+                        cudaFuncSetAttribute(fullsort_alpha_kernel<__nv_bfloat16>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kFsSmemBytes) == cudaSuccess;
+        if (dev >= 0 && ok) configured[dev] = true;
     }
     if (dtype == GR_F32)
         fullsort_alpha_kernel<float><<<batch, kFsThreads, kFsSmemBytes, st>>>((const float*)q, (const float*)p, V, n, temp_t,

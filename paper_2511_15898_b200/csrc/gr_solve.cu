@@ -546,11 +546,14 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
         if (smem > 220 * 1024) return GR_E_TOO_LARGE;
     }
     if (fa.draft && smem < kVerifyScratchBytes) smem = kVerifyScratchBytes;    // the draw's scratch
-    static int configured = 0;
-    if (configured < smem) {
+    // function attributes belong to the device: set once per device
+    static bool configured[kMaxDevices] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return GR_E_LAUNCH; }
+    if (!configured[dev]) {
         if (cudaFuncSetAttribute(solve_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess)
             return GR_E_LAUNCH;
-        configured = 220 * 1024;
+        configured[dev] = true;
     }
     solve_kernel<<<batch, kSolveThreads, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
                                                      max_iters, qstep, Qt, only_flagged, alpha_out, status_out, fa);
