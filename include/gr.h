@@ -236,6 +236,23 @@ int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, 
 int gr_read_rule(const void* params, int batch, int kcap, int* ids, int* block, double* w,
                  double* resid, double* flow, double* header, void* stream);
 
+/*
+ * gr_read_slice -- the slice pi(.|omega) of every instance for its drafted tuple (Eq. "cases" and Eq. "approx-c",
+ * "normalized" as in Algorithm 1), computed by the same device code gr_verify draws from, for inspection and tests:
+ * what gr_verify compares u0 with, without the draw.
+ *   params        written by gr_solve (not by gr_solve_verify) for the same batch; read only.
+ *   draft_tokens  [batch, n] int32, n as given to gr_solve.
+ *   U    out [batch, n] int32: U[b, s] = drafted token s of instance b, or -1 when it repeats an earlier one.
+ *   pi   out [batch, n] double: probability that token is emitted (0 for repeats, and for tokens outside the
+ *        block that serves the tuple); the accepted segments of the draw are these, in this order.
+ *   rho  out [batch] double: mass of the resample segment (1 / (1 + sum of the weights) when every drafted token
+ *        lies in H*, else 0).
+ *   status out [batch]: GR_OK / GR_NOT_CONVERGED (slice given), or GR_DRAFT_OUT_OF_SUPPORT /
+ *        GR_SUPPORT_TOO_LARGE / GR_BAD_LOGITS / GR_PARTIAL_RULE / GR_STALE_PARAMS (no slice: U = -1, pi = 0).
+ */
+int gr_read_slice(const void* params, const int* draft_tokens, int batch, int n, int* U, double* pi,
+                  double* rho, int* status, void* stream);
+
 /* Text for a GR_* / GR_E_* code (host pointer to a static string). */
 const char* gr_strerror(int code);
 

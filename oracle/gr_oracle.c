@@ -589,8 +589,12 @@ int gro_solve_verify_batch(const double *tl, const double *dl, int batch, int V,
                            const int *draft_tokens, const float *uniforms,
                            double *alpha_star, int *token, int *accepted, int *status,
                            int *U_out, double *pi_out, double *rho_out, double *gnorm_out, int *iters_out,
-                           int *jstar_out)
+                           int *jstar_out,
+                           int kcap, int *k_out, int *nblocks_out, int *order_out, int *block_out,
+                           double *w_out, double *r_out, double *p_out, double *psi_out)
 {
+    /* the last group of outputs is optional (NULL skips): the whole solution of every instance, per-support arrays
+     * with kcap entries per instance in ratio order (psi: kcap + 1), unused entries -1 / 0 */
     int k = (topk <= 0 || topk >= V) ? V : topk;
 #pragma omp parallel for schedule(dynamic, 1)
     for (int b = 0; b < batch; b++) {
@@ -609,6 +613,18 @@ int gro_solve_verify_batch(const double *tl, const double *dl, int batch, int V,
         if (gnorm_out) gnorm_out[b] = gn;
         if (iters_out) iters_out[b] = iters;
         if (jstar_out) jstar_out[b] = jstar;
+        if (k_out) k_out[b] = kk;
+        if (nblocks_out) nblocks_out[b] = nb;
+        for (int j = 0; j < kcap; j++) {
+            size_t o = (size_t)b * kcap + j;
+            int in = j < kk;
+            if (order_out) order_out[o] = in ? order[j] : -1;
+            if (block_out) block_out[o] = in ? block[j] : -2;
+            if (w_out) w_out[o] = in ? w[j] : 0.0;
+            if (r_out) r_out[o] = in ? r[j] : 0.0;
+            if (p_out) p_out[o] = in ? p[j] : 0.0;
+        }
+        if (psi_out) for (int j = 0; j <= kcap; j++) psi_out[(size_t)b * (kcap + 1) + j] = j <= kk ? psi[j] : 0.0;
         int *U = (int *)malloc(sizeof(int) * (size_t)n);
         double *pi = (double *)malloc(sizeof(double) * (size_t)n);
         double rho = 0.0;
@@ -626,6 +642,143 @@ int gro_solve_verify_batch(const double *tl, const double *dl, int batch, int V,
         if (pi_out) for (int s = 0; s < n; s++) pi_out[(size_t)b * n + s] = (nu > 0 && s < nu) ? pi[s] : 0.0;
         if (rho_out) rho_out[b] = (nu > 0) ? rho : 0.0;
         free(U); free(pi); free(tgt); free(drf); free(order); free(block); free(buf);
+    }
+    return GRO_OK;
+}
+
+/* ------------------------------------------------------------------ certificate
+ * The structure of every instance (distributions, ratio order, H*, residuals, blocks: steps O1-O5, no convex
+ * solve) and, for weights w_in given from outside (per-support arrays of kcap entries per instance in THIS
+ * ratio order), the L1 norm of the gradient of the convex functions at those weights,
+ *   || g_inner(w) - tgt ||_1 on H*  +  sum over outer blocks with >= 2 tokens of || g_block(w) - p ||_1
+ * (Thm "Inner Convex Solver", Thm "Outer Convex Solver": the gradient of Theta / Phi is g - rhs), one gradient
+ * evaluation per system by the integral route.  A small value certifies the weights: inside a system the
+ * stationary point is unique.  Weights of positions outside every solved system are ignored.
+ * lse_in (optional, NULL = none): a log-sum-exp of the target row per instance given from outside; cert2_out then
+ * receives the same norm with the target normalised by THAT value (tgt_i = exp(tl_i / Tt - lse_in)), which separates
+ * the error of the weights from the error of the normalisation they were solved for.  The structure always comes
+ * from the oracle's own distributions.
+ */
+int gro_certify_batch(const double *tl, const double *dl, int batch, int V, int n, int topk, double Tt, double Td,
+                      const double *w_in, int kcap, const double *lse_in, double *cert2_out, double *lse_out,
+                      int *k_out, int *jstar_out, int *nblocks_out, double *alpha_star_out,
+                      int *order_out, int *block_out, double *r_out, double *p_out, double *psi_out,
+                      double *cert_out)
+{
+    int k = (topk <= 0 || topk >= V) ? V : topk;
+    if (k > kcap) return GRO_BAD_ARG;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < batch; b++) {
+        const double *tlb = tl + (size_t)b * V, *dlb = dl + (size_t)b * V;
+        double *tgt = (double *)malloc(sizeof(double) * (size_t)V);
+        double *drf = (double *)malloc(sizeof(double) * (size_t)V);
+        int *ids = (int *)malloc(sizeof(int) * (size_t)V);
+        int *order = (int *)malloc(sizeof(int) * (size_t)k);
+        int *block = (int *)malloc(sizeof(int) * (size_t)k);
+        double *buf = (double *)malloc(sizeof(double) * (size_t)(8 * k + 3));
+        double *tgt_pos = buf, *drf_pos = buf + k, *psi = buf + 2 * k, *p = buf + 3 * k + 1, *r = buf + 4 * k + 1,
+               *Tg = buf + 5 * k + 1, *Dr = buf + 6 * k + 2, *g = buf + 7 * k + 3;
+        double lse_own = 0.0;
+        int kk = gro_distributions(tlb, dlb, V, topk, Tt, Td, tgt, drf, ids, &lse_own);
+        if (lse_out) lse_out[b] = lse_own;
+        double as = 0.0;
+        int jstar = gro_subset_selection(tlb, dlb, tgt, drf, ids, kk, n, Tt, Td, kk == V, order, psi, Tg, Dr, &as);
+        for (int j = 0; j < kk; j++) { tgt_pos[j] = tgt[order[j]]; drf_pos[j] = drf[order[j]]; }
+        int nb = gro_outer_residuals(tgt_pos, psi, kk, jstar, p, r, block);
+        const double *w = w_in + (size_t)b * kcap;
+        /* right-hand sides under the outside normalisation: targets rescaled, the chain psi = Tg - Dr^n and the
+         * residuals recomputed from them (block boundaries kept) */
+        double scale2 = lse_in ? exp(lse_own - lse_in[b]) : 1.0;
+        double *tgt2 = (double *)malloc(sizeof(double) * (size_t)(3 * kk + 2));
+        double *psi2 = tgt2 + kk, *p2 = psi2 + kk + 1;
+        double *r2 = (double *)malloc(sizeof(double) * (size_t)(kk + 1));
+        int *block2 = (int *)malloc(sizeof(int) * (size_t)(kk + 1));
+        for (int j = 0; j < kk; j++) tgt2[j] = tgt_pos[j] * scale2;
+        for (int j = 0; j <= kk; j++) psi2[j] = Tg[j] * scale2 - (Tg[j] - psi[j]);
+        gro_outer_residuals(tgt2, psi2, kk, jstar, p2, r2, block2);
+        double cert = 0.0, cert2 = 0.0;
+        if (jstar > 0) {
+            gro_grad_g2(jstar, drf_pos, w, n, 0.0, 1, g);
+            for (int i = 0; i < jstar; i++) { cert += fabs(g[i] - tgt_pos[i]); cert2 += fabs(g[i] - tgt_pos[i] * scale2); }
+        }
+        for (int bk = 0; bk < nb; bk++) {
+            int lo = -1, hi = -1;
+            for (int j = jstar; j < kk; j++) if (block[j] == bk) { if (lo < 0) lo = j; hi = j; }
+            if (lo < 0 || hi == lo) continue;
+            int m = hi - lo + 1;
+            gro_grad_g2(m, drf_pos + lo, w + lo, n, Dr[lo], 0, g);
+            for (int i = 0; i < m; i++) { cert += fabs(g[i] - p[lo + i]); cert2 += fabs(g[i] - p2[lo + i]); }
+        }
+        if (cert2_out) cert2_out[b] = cert2;
+        free(tgt2); free(r2); free(block2);
+        k_out[b] = kk; jstar_out[b] = jstar; nblocks_out[b] = nb; alpha_star_out[b] = as; cert_out[b] = cert;
+        for (int j = 0; j < kcap; j++) {
+            size_t o = (size_t)b * kcap + j;
+            int in = j < kk;
+            order_out[o] = in ? order[j] : -1;
+            block_out[o] = in ? block[j] : -2;
+            r_out[o] = in ? r[j] : 0.0;
+            p_out[o] = in ? p[j] : 0.0;
+        }
+        for (int j = 0; j <= kcap; j++) psi_out[(size_t)b * (kcap + 1) + j] = j <= kk ? psi[j] : 0.0;
+        free(tgt); free(drf); free(ids); free(order); free(block); free(buf);
+    }
+    return GRO_OK;
+}
+
+/* ------------------------------------------------------------------ draw sweep
+ * Many draws from one solved rule per instance (App. A steps 3-4 through gro_slice / gro_draw): for R pairs of
+ * uniforms per instance the emitted token and accepted flag, and how far the deciding uniform is from the nearest
+ * boundary of the CDF it was compared with (the parity tests excuse a differing token only within 1e-6 of one).
+ * The rule is given as per-support arrays of kcap entries per instance in ratio order (as gro_solve_verify_batch
+ * returns them); uniforms are [batch, R, 2].
+ */
+int gro_draw_sweep_batch(const double *tl, const double *dl, int batch, int V, int n, int topk, double Tt, double Td,
+                         int kcap, const int *k_in, const int *jstar_in, const int *order_in, const int *block_in,
+                         const double *w_in, const double *r_in, const int *draft_tokens, const float *uniforms, int R,
+                         int *token_out, int *accepted_out, double *margin_out)
+{
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int b = 0; b < batch; b++) {
+        const double *tlb = tl + (size_t)b * V, *dlb = dl + (size_t)b * V;
+        double *rfull = (double *)malloc(sizeof(double) * (size_t)V);
+        double *drf = (double *)malloc(sizeof(double) * (size_t)V);
+        double *cum = (double *)malloc(sizeof(double) * (size_t)V);
+        int *ids = (int *)malloc(sizeof(int) * (size_t)V);
+        int *U = (int *)malloc(sizeof(int) * (size_t)n);
+        double *pi = (double *)malloc(sizeof(double) * (size_t)n);
+        gro_distributions(tlb, dlb, V, topk, Tt, Td, rfull, drf, ids, NULL);      /* rfull = tgt for now */
+        const int kk = k_in[b];
+        const int *order = order_in + (size_t)b * kcap, *block = block_in + (size_t)b * kcap;
+        const double *w = w_in + (size_t)b * kcap, *r = r_in + (size_t)b * kcap;
+        for (int j = 0; j < kk; j++) rfull[order[j]] = r[j];
+        double tot = 0.0;
+        for (int i = 0; i < V; i++) { tot += rfull[i]; }
+        double acc = 0.0;
+        for (int i = 0; i < V; i++) { acc += rfull[i]; cum[i] = acc; }            /* same summation order as gro_draw */
+        double rho = 0.0;
+        int nu = gro_slice(kk, n, jstar_in[b], order, block, w, draft_tokens + (size_t)b * n, U, pi, &rho);
+        for (int q = 0; q < R; q++) {
+            size_t o = (size_t)b * R + q;
+            double u0 = (double)uniforms[2 * o], u1 = (double)uniforms[2 * o + 1];
+            if (nu < 0) { token_out[o] = -1; accepted_out[o] = 0; margin_out[o] = 1.0; continue; }
+            int tk = -1, ac = 0;
+            gro_draw(nu, U, pi, rho, rfull, V, u0, u1, &tk, &ac);
+            token_out[o] = tk; accepted_out[o] = ac;
+            /* distance of u0 to the edges of the accepted segments */
+            double mg = 1.0, c = 0.0;
+            for (int u = 0; u < nu; u++) { c += pi[u]; if (fabs(c - u0) < mg) mg = fabs(c - u0); }
+            if (!ac && tot > 0.0) {
+                /* resample branch: distance of u1 to the CDF edges on either side of the emitted token */
+                double thr = u1 * tot;
+                double hi = cum[tk], lo = tk > 0 ? cum[tk - 1] : 0.0;
+                double m1 = fabs(hi - thr) / tot, m0 = fabs(thr - lo) / tot;
+                double mr = m1 < m0 ? m1 : m0;
+                if (mr < mg) mg = mr;
+            }
+            margin_out[o] = mg;
+        }
+        free(rfull); free(drf); free(cum); free(ids); free(U); free(pi);
     }
     return GRO_OK;
 }

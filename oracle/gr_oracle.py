@@ -185,6 +185,15 @@ class BatchResult:
     gnorm: np.ndarray
     iters: np.ndarray
     jstar: np.ndarray
+    # the whole solution of every instance, per-support arrays [B, kcap] in ratio order (padding -1 / -2 / 0)
+    k: np.ndarray
+    nblocks: np.ndarray
+    order: np.ndarray
+    block: np.ndarray
+    w: np.ndarray
+    r: np.ndarray
+    p: np.ndarray
+    psi: np.ndarray      # [B, kcap + 1]
 
 
 def solve_verify_batch(tl, dl, n, topk, Tt, Td, draft_tokens, uniforms, route=ROUTE_G2, tol=1e-12,
@@ -196,12 +205,79 @@ def solve_verify_batch(tl, dl, n, topk, Tt, Td, draft_tokens, uniforms, route=RO
     a = np.zeros(B); token = np.zeros(B, dtype=np.int32); acc = np.zeros(B, dtype=np.int32)
     status = np.zeros(B, dtype=np.int32); U = np.zeros((B, n), dtype=np.int32); pi = np.zeros((B, n))
     rho = np.zeros(B); gn = np.zeros(B); it = np.zeros(B, dtype=np.int32); js = np.zeros(B, dtype=np.int32)
+    kcap = V if (topk <= 0 or topk >= V) else int(topk)
+    kk = np.zeros(B, dtype=np.int32); nb = np.zeros(B, dtype=np.int32)
+    order = np.zeros((B, kcap), dtype=np.int32); block = np.zeros((B, kcap), dtype=np.int32)
+    w = np.zeros((B, kcap)); r = np.zeros((B, kcap)); p = np.zeros((B, kcap)); psi = np.zeros((B, kcap + 1))
     D = C.c_double
     lib().gro_solve_verify_batch(_p(tl, D), _p(dl, D), B, V, int(n), int(topk), D(Tt), D(Td), int(route), int(method), D(tol),
                                  int(max_iter), _p(toks, C.c_int), _p(uni, C.c_float), _p(a, D), _p(token, C.c_int),
                                  _p(acc, C.c_int), _p(status, C.c_int), _p(U, C.c_int), _p(pi, D), _p(rho, D),
-                                 _p(gn, D), _p(it, C.c_int), _p(js, C.c_int))
-    return BatchResult(a, token, acc, status, U, pi, rho, gn, it, js)
+                                 _p(gn, D), _p(it, C.c_int), _p(js, C.c_int),
+                                 kcap, _p(kk, C.c_int), _p(nb, C.c_int), _p(order, C.c_int), _p(block, C.c_int),
+                                 _p(w, D), _p(r, D), _p(p, D), _p(psi, D))
+    return BatchResult(a, token, acc, status, U, pi, rho, gn, it, js, kk, nb, order, block, w, r, p, psi)
+
+
+@dataclasses.dataclass
+class Certificate:
+    k: np.ndarray
+    jstar: np.ndarray
+    nblocks: np.ndarray
+    alpha_star: np.ndarray
+    order: np.ndarray    # [B, kcap] token ids in ratio order, -1 padded
+    block: np.ndarray    # [B, kcap]
+    r: np.ndarray
+    p: np.ndarray
+    psi: np.ndarray      # [B, kcap + 1]
+    gnorm: np.ndarray    # [B] L1 gradient norm of the convex functions at the given weights
+    gnorm_lse: np.ndarray  # [B] the same with the target normalised by the log-sum-exp given from outside (nan if none)
+    lse_target: np.ndarray  # [B] the oracle's own log-sum-exp of the target row
+
+
+def certify_batch(tl, dl, n, topk, Tt, Td, w, lse=None) -> Certificate:
+    """Structure of every instance (no solve) and the L1 gradient norm at weights given from outside
+    ([B, kcap] in ratio order): one gradient evaluation per system.  `lse` ([B], optional): a target
+    log-sum-exp from outside; gnorm_lse is then the norm with the target normalised by it."""
+    tl, dl = _f64(tl), _f64(dl)
+    B, V = tl.shape
+    w = _f64(w)
+    kcap = w.shape[1]
+    kk = np.zeros(B, dtype=np.int32); js = np.zeros(B, dtype=np.int32); nb = np.zeros(B, dtype=np.int32)
+    a = np.zeros(B); cert = np.zeros(B)
+    order = np.zeros((B, kcap), dtype=np.int32); block = np.zeros((B, kcap), dtype=np.int32)
+    r = np.zeros((B, kcap)); p = np.zeros((B, kcap)); psi = np.zeros((B, kcap + 1))
+    D = C.c_double
+    cert2 = np.full(B, np.nan); lse_own = np.zeros(B)
+    lse_arr = _f64(lse) if lse is not None else None
+    st = lib().gro_certify_batch(_p(tl, D), _p(dl, D), B, V, int(n), int(topk), D(Tt), D(Td), _p(w, D), kcap,
+                                 _p(lse_arr, D) if lse_arr is not None else None,
+                                 _p(cert2, D) if lse_arr is not None else None, _p(lse_own, D),
+                                 _p(kk, C.c_int), _p(js, C.c_int), _p(nb, C.c_int), _p(a, D), _p(order, C.c_int),
+                                 _p(block, C.c_int), _p(r, D), _p(p, D), _p(psi, D), _p(cert, D))
+    if st < 0:
+        raise ValueError("bad argument")
+    return Certificate(kk, js, nb, a, order, block, r, p, psi, cert, cert2, lse_own)
+
+
+def draw_sweep_batch(tl, dl, n, topk, Tt, Td, res: BatchResult, draft_tokens, uniforms):
+    """R draws per instance from the rules in `res` (uniforms [B, R, 2]): tokens [B, R], accepted [B, R] and the
+    distance of the deciding uniform to the nearest CDF boundary [B, R]."""
+    tl, dl = _f64(tl), _f64(dl)
+    B, V = tl.shape
+    toks = _i32(draft_tokens)
+    uni = np.ascontiguousarray(uniforms, dtype=np.float32)
+    R = uni.shape[1]
+    assert uni.shape == (B, R, 2) and toks.shape == (B, n)
+    kcap = res.order.shape[1]
+    token = np.zeros((B, R), dtype=np.int32); acc = np.zeros((B, R), dtype=np.int32); margin = np.zeros((B, R))
+    D = C.c_double
+    lib().gro_draw_sweep_batch(_p(tl, D), _p(dl, D), B, V, int(n), int(topk), D(Tt), D(Td), kcap,
+                               _p(_i32(res.k), C.c_int), _p(_i32(res.jstar), C.c_int), _p(_i32(res.order), C.c_int),
+                               _p(_i32(res.block), C.c_int), _p(_f64(res.w), D), _p(_f64(res.r), D),
+                               _p(toks, C.c_int), _p(uni, C.c_float), R, _p(token, C.c_int), _p(acc, C.c_int),
+                               _p(margin, D))
+    return token, acc, margin
 
 
 def num_threads() -> int:

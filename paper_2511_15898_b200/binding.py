@@ -72,6 +72,8 @@ def load_library():
     lib.gr_verify.argtypes = [vp, ip, fp, C.c_int, ip, vp, ip, vp]
     lib.gr_read_rule.restype = C.c_int
     lib.gr_read_rule.argtypes = [vp, C.c_int, C.c_int, ip, ip, dp, dp, dp, dp, vp]
+    lib.gr_read_slice.restype = C.c_int
+    lib.gr_read_slice.argtypes = [vp, ip, C.c_int, C.c_int, ip, dp, dp, ip, vp]
     lib.gr_strerror.restype = C.c_char_p
     lib.gr_strerror.argtypes = [C.c_int]
     _lib = lib
@@ -135,6 +137,11 @@ def gr_verify(params: int, draft_tokens: int, uniforms: int, batch: int, out_tok
 def gr_read_rule(params: int, batch: int, kcap: int, ids: int, block: int, w: int, resid: int, flow: int,
                  header: int, stream: int) -> int:
     return int(load_library().gr_read_rule(params, batch, kcap, ids, block, w, resid, flow, header, stream))
+
+
+def gr_read_slice(params: int, draft_tokens: int, batch: int, n: int, U: int, pi: int, rho: int, status: int,
+                  stream: int) -> int:
+    return int(load_library().gr_read_slice(params, draft_tokens, batch, n, U, pi, rho, status, stream))
 
 
 # ---------------------------------------------------------------- torch tensors
@@ -323,6 +330,32 @@ def read_rule(solved: Solved) -> Rule:
     hd = hd.cpu()
     return Rule(ids.cpu(), blk.cpu(), w.cpu(), r.cpu(), p.cpu(), hd[:, 0].long(), hd[:, 1].long(), hd[:, 2].long(),
                 hd[:, 3], hd[:, 4], hd[:, 5].long(), hd[:, 6], hd[:, 7].long())
+
+
+@dataclasses.dataclass
+class Slice:
+    """pi(.|omega) per instance as the verification code computes it (host tensors)."""
+    U: torch.Tensor        # [B, n] int32: drafted token s, -1 for a repeat
+    pi: torch.Tensor       # [B, n] float64
+    rho: torch.Tensor      # [B] float64 mass of the resample segment
+    status: torch.Tensor   # [B] int32
+
+
+def read_slice(solved: Solved, draft_tokens: torch.Tensor) -> Slice:
+    """gr_read_slice on torch CUDA tensors."""
+    _need_cuda(draft_tokens)
+    B, n = solved.batch, solved.n
+    if draft_tokens.shape != (B, n) or draft_tokens.dtype != torch.int32:
+        raise GrError("draft_tokens must be [B, n] int32")
+    dev = draft_tokens.device
+    U = torch.empty(B, n, dtype=torch.int32, device=dev)
+    pi = torch.empty(B, n, dtype=torch.float64, device=dev)
+    rho = torch.empty(B, dtype=torch.float64, device=dev)
+    st = torch.empty(B, dtype=torch.int32, device=dev)
+    rc = gr_read_slice(solved.params.data_ptr(), draft_tokens.data_ptr(), B, n, U.data_ptr(), pi.data_ptr(),
+                       rho.data_ptr(), st.data_ptr(), _stream())
+    _check(rc, "gr_read_slice")
+    return Slice(U.cpu(), pi.cpu(), rho.cpu(), st.cpu())
 
 
 def solve_verify_host(q_logits: torch.Tensor, p_logits: torch.Tensor, draft_tokens: torch.Tensor,

@@ -174,6 +174,18 @@ int gr_read_rule(const void* params, int batch, int kcap, int* ids, int* block, 
     return GR_OK;
 }
 
+int gr_read_slice(const void* params, const int* draft_tokens, int batch, int n, int* U, double* pi, double* rho,
+                  int* status, void* stream)
+{
+    if (batch < 0 || n < 1 || n > gr::kMaxDrafts) return GR_E_INVALID;
+    if (batch == 0) return GR_OK;
+    if (!params || !draft_tokens || !U || !pi || !rho || !status) return GR_E_NULL;
+    if ((uintptr_t)params & 15) return GR_E_ALIGN;
+    gr::launch_read_slice((const char*)params, draft_tokens, batch, n, U, pi, rho, status, (cudaStream_t)stream);
+    if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    return GR_OK;
+}
+
 const char* gr_strerror(int code)
 {
     switch (code) {

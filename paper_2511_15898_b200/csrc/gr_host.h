@@ -23,6 +23,8 @@ void launch_alpha(const char* ws, int V, int topk, double temp_t, double temp_d,
                   int batch, float* alpha_out, int* status_out, cudaStream_t st);
 void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,
                    unsigned char* out_acc, int* status, cudaStream_t st);
+void launch_read_slice(const char* params, const int* draft, int batch, int n, int* U, double* pi, double* rho,
+                       int* status, cudaStream_t st);
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
                       double* flow, double* header, cudaStream_t st);
 

@@ -32,6 +32,45 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
     }
 }
 
+// The slice pi(.|omega) of every instance as the verification code computes it (one warp per instance), for
+// inspection: entry s of an instance's row belongs to drafted token s; repeats of an earlier token get id -1.
+__global__ void __launch_bounds__(kVerifyWarps * 32)
+read_slice_kernel(const char* __restrict__ params, const int* __restrict__ draft, int batch, int nmax,
+                  int* __restrict__ U, double* __restrict__ pi, double* __restrict__ rho, int* __restrict__ status_out)
+{
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    const int b = blockIdx.x * kVerifyWarps + wib;
+    if (b >= batch) return;
+    const Header* h0 = reinterpret_cast<const Header*>(params);
+    int status = GR_OK;
+    const Header* h = nullptr;
+    if (h0->magic != kMagic || h0->stride <= 0) {
+        status = GR_STALE_PARAMS;
+    } else {
+        h = reinterpret_cast<const Header*>(params + (size_t)b * h0->stride);
+        if (h->magic != kMagic) status = GR_STALE_PARAMS;
+    }
+    SliceLane sl;
+    sl.uniq = false; sl.inner = false; sl.pi = 0.0; sl.rho = 0.0;
+    int tok = -1, n = 0;
+    if (status == GR_OK) {
+        n = h->n < nmax ? h->n : nmax;
+        status = h->status;
+        if (status == GR_OK || status == GR_NOT_CONVERGED) {
+            ParamView pv = view_params((void*)h, h->kcap);
+            tok = lane < h->n ? draft[(size_t)b * h->n + lane] : -1;
+            const int rs = h->k > 0 ? slice_instance(h, pv, tok, lane, sl) : GR_SUPPORT_TOO_LARGE;
+            if (rs != GR_OK) { status = rs; sl.uniq = false; sl.pi = 0.0; sl.rho = 0.0; }
+        }
+    }
+    if (lane < nmax) {
+        const bool on = lane < n && sl.uniq;
+        U[(size_t)b * nmax + lane] = on ? tok : -1;
+        pi[(size_t)b * nmax + lane] = on ? sl.pi : 0.0;
+    }
+    if (lane == 0) { rho[b] = sl.rho; status_out[b] = status; }
+}
+
 // copies the rule out of the params block into plain arrays
 __global__ void read_rule_kernel(const char* __restrict__ params, int batch, int kcap_out, int* ids, int* block,
                                  double* w, double* resid, double* flow, double* header)
@@ -66,6 +105,12 @@ void launch_verify(const char* params, const int* draft, const float* uni, int b
 {
     const int blocks = (batch + kVerifyWarps - 1) / kVerifyWarps;
     verify_kernel<<<blocks, kVerifyWarps * 32, 0, st>>>(params, draft, uni, batch, out_token, out_acc, status);
+}
+void launch_read_slice(const char* params, const int* draft, int batch, int n, int* U, double* pi, double* rho,
+                       int* status, cudaStream_t st)
+{
+    const int blocks = (batch + kVerifyWarps - 1) / kVerifyWarps;
+    read_slice_kernel<<<blocks, kVerifyWarps * 32, 0, st>>>(params, draft, batch, n, U, pi, rho, status);
 }
 void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* block, double* w, double* resid,
                       double* flow, double* header, cudaStream_t st)

@@ -131,30 +131,17 @@ __device__ inline int resample_draw(const Header* h, const ParamView& pv, int k,
 }
 
 
-// The whole verification of one instance by one warp.  `h` is the instance's header (already checked to carry
-// the magic number); a rule marked partial is accepted only from the kernel that solved it for these drafts.
-__device__ inline void verify_instance(const Header* h, const int* draft_row, const float* uni_row, int lane,
-                                       const VerifyScratch& vs, bool allow_partial, int& token, int& accepted,
-                                       int& status)
+// One lane's share of the slice pi(.|omega) (Eq. "cases", Eq. "approx-c", "normalized" in Algorithm 1): lane s < n
+// holds drafted token s.  uniq: first occurrence of its token; pi: its probability (0 for repeats and for tokens
+// outside the serving system); inner: every drafted token lies in H*; rho: mass of the resample segment.
+struct SliceLane { bool uniq, inner; double pi, rho; };
+
+// Slice of a solved instance (k > 0) for the drafted tuple, one warp; `tok` is this lane's drafted token (lanes >= n: any).
+// Returns GR_OK, or GR_DRAFT_OUT_OF_SUPPORT when a drafted token is not in the support.
+__device__ inline int slice_instance(const Header* h, const ParamView& pv, int tok, int lane, SliceLane& sl)
 {
-    token = -1; accepted = 0;
-    status = h->status;
-    if (status == GR_BAD_LOGITS) return;
-    if (status == GR_PARTIAL_RULE) {
-        if (!allow_partial) return;
-        status = GR_OK;
-    }
-    ParamView pv = view_params((void*)h, h->kcap);
     const int n = h->n, k = h->k, jstar = h->jstar;
-    const double u0 = (double)uni_row[0], u1 = (double)uni_row[1];
-    const int tok = lane < n ? draft_row[lane] : -1;
-    if (k == 0) {
-        // no rule was solved: emit a sample of the target distribution itself
-        token = resample_draw(h, pv, 0, u1, lane, vs.l_id, vs.l_r, vs.s_id, vs.s_p);
-        accepted = __any_sync(0xffffffffu, lane < n && tok == token) ? 1 : 0;
-        if (token < 0) accepted = 0;
-        return;
-    }
+    sl.uniq = false; sl.inner = false; sl.pi = 0.0; sl.rho = 0.0;
     // position of every drafted token in the ratio order
     int pos = -1;
     for (int s = 0; s < n; s++) {
@@ -168,7 +155,7 @@ __device__ inline void verify_instance(const Header* h, const int* draft_row, co
         if (lane == s) pos = found;
     }
     const bool missing = __any_sync(0xffffffffu, lane < n && pos < 0);
-    if (missing) { status = GR_DRAFT_OUT_OF_SUPPORT; return; }
+    if (missing) return GR_DRAFT_OUT_OF_SUPPORT;
     // distinct tokens in order of first occurrence; the lowest-ratio position met
     bool uniq = lane < n;
     int maxpos = lane < n ? pos : -1;
@@ -184,7 +171,40 @@ __device__ inline void verify_instance(const Header* h, const int* draft_row, co
         else wv = (pv.blk[pos] == pv.blk[maxpos]) ? pv.w[pos] : 0.0;
     }
     const double W = warp_sum(wv) + (inner ? 1.0 : 0.0);
-    const double pi = wv / W;
+    sl.uniq = uniq; sl.inner = inner;
+    sl.pi = wv / W;
+    sl.rho = inner ? 1.0 / W : 0.0;
+    return GR_OK;
+}
+
+// The whole verification of one instance by one warp.  `h` is the instance's header (already checked to carry
+// the magic number); a rule marked partial is accepted only from the kernel that solved it for these drafts.
+__device__ inline void verify_instance(const Header* h, const int* draft_row, const float* uni_row, int lane,
+                                       const VerifyScratch& vs, bool allow_partial, int& token, int& accepted,
+                                       int& status)
+{
+    token = -1; accepted = 0;
+    status = h->status;
+    if (status == GR_BAD_LOGITS) return;
+    if (status == GR_PARTIAL_RULE) {
+        if (!allow_partial) return;
+        status = GR_OK;
+    }
+    ParamView pv = view_params((void*)h, h->kcap);
+    const int n = h->n, k = h->k;
+    const double u0 = (double)uni_row[0], u1 = (double)uni_row[1];
+    const int tok = lane < n ? draft_row[lane] : -1;
+    if (k == 0) {
+        // no rule was solved: emit a sample of the target distribution itself
+        token = resample_draw(h, pv, 0, u1, lane, vs.l_id, vs.l_r, vs.s_id, vs.s_p);
+        accepted = __any_sync(0xffffffffu, lane < n && tok == token) ? 1 : 0;
+        if (token < 0) accepted = 0;
+        return;
+    }
+    SliceLane sl;
+    if (slice_instance(h, pv, tok, lane, sl) != GR_OK) { status = GR_DRAFT_OUT_OF_SUPPORT; return; }
+    const bool uniq = sl.uniq, inner = sl.inner;
+    const double pi = sl.pi;
     const double cum = warp_incl_scan(pi, lane);
     const unsigned hit = __ballot_sync(0xffffffffu, uniq && cum > u0);
     if (hit) {

@@ -1,15 +1,25 @@
 """GPU-vs-oracle comparison used by the parity tests (and nothing else).
 
 `compare(wl)` runs the CUDA path through the C interface on a workload, runs the fp64
-CPU oracle on the same tensors, and returns the figures the tolerances are stated on:
+CPU oracle on the same tensors (one solve per instance, in C, OpenMP over instances), and
+returns the figures the tolerances are stated on:
   alpha_err      max |alpha*_gpu - alpha*_oracle|
   tv             max total-variation distance between the two verification
-                 distributions pi(.|omega) for the drafted omega (accepted tokens,
-                 resample mass, and the resample distribution on the support)
-  token_mismatch instances whose emitted token differs, split into draws within 1e-6
-                 of a CDF boundary (excused) and others (failures)
+                 distributions pi(.|omega) for the drafted omega; the GPU side is what the
+                 verification device code itself computes (gr_read_slice) for the accepted
+                 tokens and the resample mass, and the rule's residuals for the resample
+                 distribution on the support
+  token_mismatch draws whose emitted token differs, split into draws within 1e-6
+                 of a CDF boundary (excused) and others (failures); with `draws` > 1 every
+                 instance is drawn that many times (fresh seeded uniforms, a share of them
+                 forced past the accepted mass so that the resample branch runs)
 Instances whose discrete structure (|H*|, block boundaries) hinges on a gap below
 `tie_gap` in the oracle's psi chain are counted and left out of the tv / token figures.
+
+`certify(wl)` checks EVERY instance of a batch without solving it on the CPU: the oracle
+recomputes the structure and evaluates the gradient of the convex functions once at the
+GPU's weights (the stationary point of each system is unique, so a small gradient norm
+pins the weights).
 """
 from __future__ import annotations
 
@@ -37,6 +47,7 @@ class Report:
     token_mismatch_boundary: int
     token_mismatch_other: int
     n_tokens_compared: int
+    n_resampled: int            # compared draws that took the resample branch (oracle side)
     accept_rate_gpu: float
     accept_rate_oracle: float
     details: list
@@ -46,121 +57,208 @@ class Report:
                 f"gnorm={self.gnorm_max:.2e} iters<={self.iters_max} notconv={self.n_not_converged} "
                 f"near_tie={self.n_near_tie} struct_mismatch={self.n_struct_mismatch} "
                 f"tok_mismatch(boundary/other)={self.token_mismatch_boundary}/{self.token_mismatch_other} of "
-                f"{self.n_tokens_compared} acc(gpu/oracle)={self.accept_rate_gpu:.4f}/{self.accept_rate_oracle:.4f}")
+                f"{self.n_tokens_compared} draws ({self.n_resampled} resampled) "
+                f"acc(gpu/oracle)={self.accept_rate_gpu:.4f}/{self.accept_rate_oracle:.4f}")
 
 
-def _near_tie(sol: "O.Solution", gap: float) -> bool:
+def near_tie(psi: np.ndarray, k: int, jstar: int, V: int, gap: float) -> bool:
     """True when |H*| or a block boundary is decided by a psi difference below `gap`.
     The closing value psi(whole support) = 0 of an untruncated draft is set exactly on both
     sides, so its tie with psi(empty) = 0 is not a rounding matter and does not count."""
-    psi = sol.psi[: sol.k + 1]
-    best = psi[sol.jstar]
-    drop = [sol.jstar]
-    if sol.k == sol.V and sol.jstar == 0:
-        drop.append(sol.k)
+    psi = psi[: k + 1]
+    best = psi[jstar]
+    drop = [jstar]
+    if k == V and jstar == 0:
+        drop.append(k)
     others = np.delete(psi, drop)
     if others.size and np.min(np.abs(others - best)) < gap:
         return True
-    m_prev = psi[sol.k]
-    for s in range(1, sol.k - sol.jstar + 1):
-        c = psi[sol.k - s]
+    m_prev = psi[k]
+    for s in range(1, k - jstar + 1):
+        c = psi[k - s]
         if abs(c - m_prev) < gap and not (c == m_prev):
             return True
         m_prev = min(m_prev, c)
     return False
 
 
-def _slice_from_rule(ids, blk, w, jstar, omega):
-    """pi(.|omega) on the distinct drafted tokens and the resample mass, from a rule in ratio order."""
-    pos = []
-    U = []
-    idl = ids.tolist()
-    for t in omega.tolist():
-        if t not in idl:
-            return None
-        p = idl.index(t)
-        if p not in pos:
-            pos.append(p); U.append(t)
-    mp = max(pos)
-    if mp < jstar:
-        ww = np.array([w[p] for p in pos])
-        Wt = 1.0 + ww.sum()
-        return U, ww / Wt, 1.0 / Wt
-    b = blk[mp]
-    ww = np.array([w[p] if blk[p] == b else 0.0 for p in pos])
-    return U, ww / ww.sum(), 0.0
+def _host_inputs(wl: W.Workload):
+    return (W.logits_to_f64(wl.q_logits), W.logits_to_f64(wl.p_logits), wl.draft_tokens.cpu().numpy(),
+            wl.uniforms.cpu().numpy())
+
+
+def _sweep_uniforms(B: int, draws: int, rho: np.ndarray, seed: int) -> np.ndarray:
+    """[B, draws, 2] float32: the first half uniform in the unit square; the second half with u0 placed inside the
+    resample segment where there is one (so that the two-level residual CDF is exercised by every instance that has
+    it), u1 uniform, plus a grid of u1 values across the whole row."""
+    rng = np.random.default_rng(seed)
+    u = rng.random((B, draws, 2)).astype(np.float32)
+    half = draws // 2
+    if half:
+        lo = (1.0 - rho)[:, None]
+        forced = lo + rho[:, None] * rng.random((B, draws - half))
+        u[:, half:, 0] = np.where(rho[:, None] > 1e-6, np.minimum(forced, 1.0 - 1e-7), u[:, half:, 0]).astype(np.float32)
+        grid = (np.arange(draws - half) + 0.5) / (draws - half)
+        u[:, half:, 1] = grid[None, :].astype(np.float32)
+    return np.clip(u, 0.0, np.float32(1.0 - 2.0 ** -24))
 
 
 def compare(wl: W.Workload, opt=None, oracle_tol: float = 1e-11, tie_gap: float = 1e-6,
-            boundary: float = 1e-6) -> Report:
+            boundary: float = 1e-6, draws: int = 1, fused: bool = False) -> Report:
+    """`fused`: the emitted tokens come from gr_solve_verify (one call) instead of gr_solve + gr_verify; the rule
+    and the slice are still read from a two-call solve of the same inputs."""
     assert wl.q_logits.is_cuda
+    B, n = wl.batch, wl.n
     solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft, opt)
-    ver = G.verify(solved, wl.draft_tokens, wl.uniforms)
     rule = G.read_rule(solved)
+    sl = G.read_slice(solved, wl.draft_tokens)
     torch.cuda.synchronize()
     g_alpha = solved.alpha_star.cpu().numpy().astype(np.float64)
-    g_tok = ver.token.cpu().numpy(); g_acc = ver.accepted.cpu().numpy().astype(np.int32)
-    g_st = ver.status.cpu().numpy()
 
-    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
-    toks = wl.draft_tokens.cpu().numpy(); uni = wl.uniforms.cpu().numpy()
-    B = wl.batch
+    tl, dl, toks, uni = _host_inputs(wl)
     res = O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, toks, uni, tol=oracle_tol)
+
+    # draws: the workload's own uniforms first, then the seeded sweep
+    U = np.empty((B, draws, 2), dtype=np.float32)
+    U[:, 0, :] = uni
+    if draws > 1:
+        U[:, 1:, :] = _sweep_uniforms(B, draws - 1, res.rho, seed=wl.V * 31 + B)
+    g_tok = np.empty((B, draws), dtype=np.int64); g_acc = np.empty((B, draws), dtype=np.int64)
+    g_st = None
+    for q in range(draws):
+        uq = torch.from_numpy(np.ascontiguousarray(U[:, q, :])).to(wl.q_logits.device)
+        if fused:
+            _, ver = G.solve_verify(wl.q_logits, wl.p_logits, wl.draft_tokens, uq, wl.topk, wl.temp_target,
+                                    wl.temp_draft, opt)
+        else:
+            ver = G.verify(solved, wl.draft_tokens, uq)
+        torch.cuda.synchronize()
+        g_tok[:, q] = ver.token.cpu().numpy(); g_acc[:, q] = ver.accepted.cpu().numpy()
+        if q == 0:
+            g_st = ver.status.cpu().numpy()
+    o_tok, o_acc, margin = O.draw_sweep_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, res, toks, U)
+    assert np.array_equal(o_tok[:, 0], res.token) and np.array_equal(o_acc[:, 0], res.accepted)
 
     alpha_err = float(np.max(np.abs(g_alpha - res.alpha_star))) if B else 0.0
     alpha_err = max(alpha_err, float(np.max(np.abs(rule.alpha_star.numpy() - res.alpha_star))) if B else 0.0)
     tv_max = 0.0; wrel = 0.0
-    near = 0; struct_bad = 0; mm_b = 0; mm_o = 0; ncmp = 0
+    near = 0; struct_bad = 0; mm_b = 0; mm_o = 0; ncmp = 0; nres = 0
     details = []
+    g_ids = rule.ids.numpy(); g_blk = rule.block.numpy(); g_w = rule.w.numpy(); g_r = rule.resid.numpy()
+    s_U = sl.U.numpy(); s_pi = sl.pi.numpy(); s_rho = sl.rho.numpy(); s_st = sl.status.numpy()
     for b in range(B):
-        sol = O.solve(tl[b], dl[b], wl.n, wl.topk, wl.temp_target, wl.temp_draft, tol=oracle_tol)
-        k = sol.k
-        ids = rule.ids[b, :k].numpy(); blk = rule.block[b, :k].numpy(); w = rule.w[b, :k].numpy()
-        rr = rule.resid[b, :k].numpy()
-        if _near_tie(sol, tie_gap):
+        k = int(res.k[b]); js = int(res.jstar[b])
+        if near_tie(res.psi[b], k, js, wl.V, tie_gap):
             near += 1
             continue
-        same = (int(rule.k[b]) == k and int(rule.jstar[b]) == sol.jstar and np.array_equal(ids, sol.order)
-                and np.array_equal(blk, sol.block))
+        ids = g_ids[b, :k]; blk = g_blk[b, :k]; w = g_w[b, :k]; rr = g_r[b, :k]
+        o_blk = res.block[b, :k]
+        same = (int(rule.k[b]) == k and int(rule.jstar[b]) == js and np.array_equal(ids, res.order[b, :k])
+                and np.array_equal(blk, o_blk))
         if not same:
             struct_bad += 1
-            details.append((b, "structure", int(rule.jstar[b]), sol.jstar))
+            details.append((b, "structure", int(rule.jstar[b]), js))
             continue
         # weights: compare scale-free inside outer blocks
-        wo = sol.w.copy(); wg = w.copy()
+        wo = res.w[b, :k].copy(); wg = w.copy()
         for bk in set(blk.tolist()):
             if bk < 0:
                 continue
             sel = blk == bk
             wo[sel] /= np.exp(np.mean(np.log(wo[sel]))); wg[sel] /= np.exp(np.mean(np.log(wg[sel])))
         wrel = max(wrel, float(np.max(np.abs(wg / wo - 1.0))))
-        sl_g = _slice_from_rule(ids, blk, w, sol.jstar, toks[b])
-        nu, U, pi_o, rho_o = O.slice_(sol, toks[b])
-        assert sl_g is not None and nu > 0
-        Ug, pi_g, rho_g = sl_g
-        assert list(Ug) == list(U)
+        if res.status[b] < 0:
+            # a drafted token outside the support: both sides must say so
+            assert s_st[b] == G.GR_DRAFT_OUT_OF_SUPPORT and g_st[b] == G.GR_DRAFT_OUT_OF_SUPPORT
+            continue
+        # the kernel's slice against the oracle's: distinct drafted tokens in first-occurrence order
+        assert s_st[b] in (G.GR_OK, G.GR_NOT_CONVERGED), (b, int(s_st[b]))
+        keep = s_U[b] >= 0
+        Ug = s_U[b][keep]; pi_g = s_pi[b][keep]; rho_g = float(s_rho[b])
+        nu = int((res.U[b] >= 0).sum())
+        assert list(Ug) == list(res.U[b, :nu]), (b, Ug, res.U[b])
+        pi_o = res.pi[b, :nu]; rho_o = float(res.rho[b])
         # total variation over emitted tokens: accepted part + resample part (rho * res(.))
-        res_o = sol.r / max(1.0 - sol.alpha_star, 1e-300)
-        res_g = rr / max(1.0 - float(rule.alpha_star[b]), 1e-300)
+        a_o = float(res.alpha_star[b]); a_g = float(rule.alpha_star[b])
+        res_o = res.r[b, :k] / max(1.0 - a_o, 1e-300)
+        res_g = rr / max(1.0 - a_g, 1e-300)
         tv = 0.5 * (np.abs(pi_g - pi_o).sum() + np.abs(rho_g * res_g - rho_o * res_o).sum()
                     + abs(rho_g * (1 - res_g.sum()) - rho_o * (1 - res_o.sum())))
         tv_max = max(tv_max, float(tv))
-        # emitted token
-        ncmp += 1
-        if g_tok[b] != res.token[b] or g_acc[b] != res.accepted[b]:
-            u0, u1 = float(uni[b, 0]), float(uni[b, 1])
-            edges = np.concatenate([np.cumsum(pi_o)])
-            close = bool(np.min(np.abs(edges - u0)) < boundary)
-            if not close and rho_o > 0:
-                rfull = sol.residual_full()
-                cdf = np.cumsum(rfull) / rfull.sum()
-                close = bool(np.min(np.abs(cdf - u1)) < boundary)
-            if close:
-                mm_b += 1
-            else:
-                mm_o += 1
-                details.append((b, "token", int(g_tok[b]), int(res.token[b]), int(g_acc[b]), int(res.accepted[b])))
+        # emitted tokens
+        for q in range(draws):
+            ncmp += 1
+            nres += int(o_acc[b, q] == 0)
+            if g_tok[b, q] != o_tok[b, q] or g_acc[b, q] != o_acc[b, q]:
+                if margin[b, q] < boundary:
+                    mm_b += 1
+                else:
+                    mm_o += 1
+                    details.append((b, "token", q, int(g_tok[b, q]), int(o_tok[b, q]), int(g_acc[b, q]),
+                                    int(o_acc[b, q]), float(margin[b, q])))
     ok = g_st != G.GR_DRAFT_OUT_OF_SUPPORT
     return Report(B, alpha_err, near, struct_bad, tv_max, wrel, float(rule.gnorm.max()) if B else 0.0,
                   int(rule.iters.max()) if B else 0, int((rule.status == G.GR_NOT_CONVERGED).sum()), mm_b, mm_o, ncmp,
-                  float(g_acc[ok].mean()) if B else 0.0, float(res.accepted.mean()) if B else 0.0, details)
+                  nres, float(g_acc[ok, 0].mean()) if B else 0.0, float(res.accepted.mean()) if B else 0.0, details)
+
+
+@dataclasses.dataclass
+class CertReport:
+    n_inst: int
+    n_near_tie: int
+    n_struct_mismatch: int
+    alpha_err: float
+    cert_max: float          # largest oracle-evaluated L1 gradient norm at the GPU's weights, against the oracle's own target
+    cert_solver_max: float   # the same against the target normalised by the GPU's log-sum-exp: the weights' own error
+    lse_err_max: float       # largest |lse_gpu - lse_oracle| of the target row: the normalisation's error
+    gnorm_reported_max: float
+    n_underreported: int     # instances whose reported norm is more than 10x below the solver certificate, where that is above 1e-8
+    n_status_ok: int
+    details: list
+
+    def summary(self) -> str:
+        return (f"inst={self.n_inst} near_tie={self.n_near_tie} struct_mismatch={self.n_struct_mismatch} "
+                f"alpha_err={self.alpha_err:.2e} certificate max={self.cert_max:.2e} of which weights "
+                f"{self.cert_solver_max:.2e}, target log-sum-exp error max {self.lse_err_max:.2e} "
+                f"(reported max {self.gnorm_reported_max:.2e}, under-reported {self.n_underreported}) "
+                f"status ok {self.n_status_ok}")
+
+
+def certify(wl: W.Workload, opt=None, tie_gap: float = 1e-6, chunk: int = 256) -> CertReport:
+    """Every instance of the batch: structure equal to the oracle's, and the oracle's gradient norm at the GPU's
+    weights.  The host copies of the logits are taken `chunk` rows at a time."""
+    assert wl.q_logits.is_cuda
+    solved = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft, opt)
+    rule = G.read_rule(solved)
+    torch.cuda.synchronize()
+    B = wl.batch
+    g_ids = rule.ids.numpy(); g_blk = rule.block.numpy(); g_w = rule.w.numpy(); g_lse = rule.lse_target.numpy()
+    near = 0; bad = 0; cert_max = 0.0; cert2_max = 0.0; lse_err = 0.0; alpha_err = 0.0; under = 0
+    details = []
+    for c0 in range(0, B, chunk):
+        c1 = min(B, c0 + chunk)
+        tl = W.logits_to_f64(wl.q_logits[c0:c1]); dl = W.logits_to_f64(wl.p_logits[c0:c1])
+        cert = O.certify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, g_w[c0:c1], lse=g_lse[c0:c1])
+        for i in range(c1 - c0):
+            b = c0 + i
+            k = int(cert.k[i]); js = int(cert.jstar[i])
+            alpha_err = max(alpha_err, abs(float(rule.alpha_star[b]) - float(cert.alpha_star[i])))
+            if near_tie(cert.psi[i], k, js, wl.V, tie_gap):
+                near += 1
+                continue
+            same = (int(rule.k[b]) == k and int(rule.jstar[b]) == js and np.array_equal(g_ids[b, :k], cert.order[i, :k])
+                    and np.array_equal(g_blk[b, :k], cert.block[i, :k]))
+            if not same:
+                bad += 1
+                details.append((b, "structure", int(rule.jstar[b]), js))
+                continue
+            cert_max = max(cert_max, float(cert.gnorm[i]))
+            cert2_max = max(cert2_max, float(cert.gnorm_lse[i]))
+            lse_err = max(lse_err, abs(float(g_lse[b]) - float(cert.lse_target[i])))
+            # (the kernel's quadrature resolves the norm to a few 1e-9 at its default step: smaller reported values,
+            # predictions of the last step's residual among them, are not told apart from that floor)
+            if float(cert.gnorm_lse[i]) > max(10.0 * float(rule.gnorm[b]), 1e-8):
+                under += 1
+                details.append((b, "gnorm", float(rule.gnorm[b]), float(cert.gnorm_lse[i])))
+    return CertReport(B, near, bad, alpha_err, cert_max, cert2_max, lse_err, float(rule.gnorm.max()), under,
+                      int((rule.status == G.GR_OK).sum()), details)

@@ -18,6 +18,8 @@ pytestmark = pytest.mark.gpu
 
 ALPHA_TOL = 1e-6
 TV_TOL = 1e-5
+CERT_TOL = 1e-7     # L1 gradient norm of the convex functions at the GPU's weights, evaluated by the oracle
+LSE_TOL = 1e-6      # log-sum-exp of the target row (it enters alpha* one to one, so alpha*'s tolerance applies)
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -26,36 +28,88 @@ def _lib():
     G.load_library()
 
 
-def _check(rep: P.Report, max_near_tie_frac=0.25):
+def _check(rep: P.Report, max_near_tie_frac=0.02):
+    """Near-ties (structure decided by a psi gap below 1e-6) have not been seen on any of the workloads; the
+    allowance is two in a hundred so that a rare one does not fail the suite, and the count is printed."""
     print(rep.summary())
     assert rep.alpha_err <= ALPHA_TOL, rep.summary()
     assert rep.n_struct_mismatch == 0, (rep.summary(), rep.details[:5])
     assert rep.tv <= TV_TOL, rep.summary()
     assert rep.token_mismatch_other == 0, (rep.summary(), rep.details[:5])
     assert rep.n_not_converged == 0, rep.summary()
-    assert rep.n_near_tie <= max_near_tie_frac * rep.n_inst, rep.summary()
+    assert rep.n_near_tie <= max(1, int(max_near_tie_frac * rep.n_inst)), rep.summary()
+
+
+def _check_cert(rep: P.CertReport, max_near_tie_frac=0.02):
+    print(rep.summary())
+    assert rep.alpha_err <= ALPHA_TOL, rep.summary()
+    assert rep.n_struct_mismatch == 0, (rep.summary(), rep.details[:5])
+    # the weights, for the normalisation the GPU solved them under, and that normalisation (an fp32 sum over the
+    # whole row) separately; together they bound the norm against the oracle's own target
+    assert rep.cert_solver_max <= CERT_TOL, (rep.summary(), rep.details[:5])
+    assert rep.lse_err_max <= LSE_TOL, rep.summary()
+    assert rep.cert_max <= CERT_TOL + LSE_TOL, (rep.summary(), rep.details[:5])
+    assert rep.n_underreported == 0, (rep.summary(), rep.details[:5])
+    assert rep.n_status_ok == rep.n_inst, rep.summary()
+    assert rep.n_near_tie <= max(1, int(max_near_tie_frac * rep.n_inst)), rep.summary()
 
 
 def test_config1_tiny_full_support():
-    _check(P.compare(W.config1(device="cuda")))
+    _check(P.compare(W.config1(device="cuda"), draws=64))
 
 
 def test_config2_top8():
-    _check(P.compare(W.config2(batch=64, device="cuda")))
+    rep = P.compare(W.config2(batch=128, device="cuda"), draws=64)
+    _check(rep)
+    assert rep.n_resampled > 1000          # the resample branch (two-level residual CDF) was drawn from
 
 
 def test_config3_headline_shape():
-    _check(P.compare(W.config3(batch=24, device="cuda")))
+    rep = P.compare(W.config3(batch=128, device="cuda"), draws=64)
+    _check(rep)
+    assert rep.n_resampled > 1000
 
 
 @pytest.mark.parametrize("n,topk,sigma", [(2, 5, 0.25), (4, 20, 1.0), (8, 5, 2.0), (16, 20, 0.25), (32, 5, 1.0),
                                           (32, 20, 2.0)])
 def test_config4_topk_cells(n, topk, sigma):
-    _check(P.compare(W.config4(n, topk, sigma, batch=12, device="cuda")))
+    _check(P.compare(W.config4(n, topk, sigma, batch=48, device="cuda"), draws=16))
 
 
 def test_config5_bf16_top100():
-    _check(P.compare(W.config5(batch=4, device="cuda", rows_per_pass=4)))
+    rep = P.compare(W.config5(batch=64, device="cuda", rows_per_pass=16), draws=32)
+    _check(rep)
+    assert rep.n_resampled > 500
+
+
+# ---- every instance of a whole batch: structure, and the oracle's gradient norm at the GPU's weights
+
+def test_certificate_config3_whole_batch():
+    _check_cert(P.certify(W.config3(batch=1024, device="cuda")))
+
+
+def test_certificate_config2_whole_batch():
+    _check_cert(P.certify(W.config2(batch=256, device="cuda")))
+
+
+def test_certificate_config5_512_instances():
+    _check_cert(P.certify(W.config5(batch=512, device="cuda", rows_per_pass=64), chunk=128))
+
+
+@pytest.mark.parametrize("n,topk,sigma", [(2, 20, 1.0), (8, 20, 0.25), (16, 5, 2.0), (32, 20, 1.0)])
+def test_certificate_config4_cells(n, topk, sigma):
+    _check_cert(P.certify(W.config4(n, topk, sigma, batch=512, device="cuda")))
+
+
+# ---- the one-call entry against the oracle's tokens
+
+@pytest.mark.parametrize("cfg", ["config2", "config3", "config4", "config5"])
+def test_fused_call_emits_the_oracle_tokens(cfg):
+    wl = {"config2": lambda: W.config2(batch=48, device="cuda"),
+          "config3": lambda: W.config3(batch=48, device="cuda", seed=3007),
+          "config4": lambda: W.config4(8, 20, 1.0, batch=48, device="cuda"),
+          "config5": lambda: W.config5(batch=16, device="cuda", rows_per_pass=16)}[cfg]()
+    _check(P.compare(wl, draws=8, fused=True))
 
 
 @pytest.mark.parametrize("n,topk", [(3, 70), (6, 80), (8, 128), (12, 90), (16, 128)])
@@ -176,6 +230,22 @@ def test_adversarial_row_order_takes_the_exact_selection_path():
     wl = W.Workload("adversarial", V, n, k, 1.0, 1.0, q.contiguous(), p.contiguous(), toks.contiguous(),
                     wl0.uniforms)
     _check(P.compare(wl), max_near_tie_frac=1.0)
+
+
+def test_signed_zeros_at_the_top_k_cut_tie_by_id():
+    """-0.0 and +0.0 are equal logits: the smaller id is kept whatever the sign (the oracle's comparator ties them)."""
+    V, n, k, B = 3000, 3, 6, 2
+    g = torch.Generator(device="cuda"); g.manual_seed(9)
+    q = torch.randn(B, V, generator=g, device="cuda")
+    p = -torch.rand(B, V, generator=g, device="cuda") - 0.5
+    p[:, 100:104] = 1.0                    # four clear winners
+    p[0, 7] = 0.0; p[0, 9] = -0.0; p[0, 11] = 0.0; p[0, 13] = -0.0        # the cut falls among four zeros
+    p[1, 20] = -0.0; p[1, 25] = 0.0; p[1, 30] = -0.0
+    solved = G.solve(q.contiguous(), p.contiguous(), n, k)
+    rule = G.read_rule(solved)
+    torch.cuda.synchronize()
+    assert sorted(rule.ids[0, :k].tolist()) == [7, 9, 100, 101, 102, 103]
+    assert sorted(rule.ids[1, :k].tolist()) == [20, 25, 100, 101, 102, 103]
 
 
 def test_repeat_calls_reuse_buffers_and_agree():
