@@ -456,13 +456,72 @@ int gro_newton(int route, int m, const double *d, const double *rhs, int n, doub
     return status;
 }
 
+/* ------------------------------------------------------------------ truncation sets
+ * Sec. 6.2 (tunable errors), Sec. 6.3 and Algorithm 1: the convex functions are minimised over a truncation
+ * set T only, chosen minimal with
+ *   inner:  T subset of H*,      gamma_T   = drf(H*)^n - drf(T)^n      <= tau,
+ *   outer:  T subset of V \ H*,  epsilon_T = 1 - (drf(H*) + drf(T))^n  <= tau.
+ * Fewest tokens for a given draft mass: tokens are taken in decreasing drf (equal drf: smaller id first) until
+ * the bound holds; zero-draft ids never enter.  tau <= 0 keeps every support token (both errors zero).
+ * Arrays are in ratio order (positions 0..jstar-1 = H*); in_T[pos] = 1 / 0.
+ */
+typedef struct { double d; int id; int pos; } tr_t;
+static int cmp_tr(const void *a, const void *b)
+{
+    const tr_t *x = (const tr_t *)a, *y = (const tr_t *)b;
+    if (x->d > y->d) return -1;
+    if (x->d < y->d) return 1;
+    return (x->id < y->id) ? -1 : (x->id > y->id);
+}
+int gro_truncation_sets(int k, int jstar, const int *order, const double *drf_pos, int n, double tau, int *in_T,
+                        double *gamma_out, double *eps_out)
+{
+    double D = 0.0;
+    for (int j = 0; j < jstar; j++) D += drf_pos[j];
+    double Dn = pow(D, (double)n);
+    if (!(tau > 0.0)) {
+        for (int j = 0; j < k; j++) in_T[j] = 1;
+        if (gamma_out) *gamma_out = 0.0;
+        if (eps_out) *eps_out = 0.0;
+        return GRO_OK;
+    }
+    tr_t *t = (tr_t *)malloc(sizeof(tr_t) * (size_t)(k > 0 ? k : 1));
+    for (int j = 0; j < k; j++) in_T[j] = 0;
+    /* inner */
+    for (int j = 0; j < jstar; j++) { t[j].d = drf_pos[j]; t[j].id = order[j]; t[j].pos = j; }
+    qsort(t, (size_t)jstar, sizeof(tr_t), cmp_tr);
+    double c = 0.0, gam = Dn;
+    for (int j = 0; j < jstar && gam > tau; j++) {
+        c += t[j].d; in_T[t[j].pos] = 1;
+        gam = Dn - pow(c, (double)n);
+    }
+    if (gamma_out) *gamma_out = gam > 0.0 ? gam : 0.0;
+    /* outer */
+    int mo = k - jstar;
+    for (int j = 0; j < mo; j++) { t[j].d = drf_pos[jstar + j]; t[j].id = order[jstar + j]; t[j].pos = jstar + j; }
+    qsort(t, (size_t)mo, sizeof(tr_t), cmp_tr);
+    c = D;
+    double eps = 1.0 - Dn;
+    for (int j = 0; j < mo && eps > tau; j++) {
+        c += t[j].d; in_T[t[j].pos] = 1;
+        eps = 1.0 - pow(c, (double)n);
+    }
+    if (eps_out) *eps_out = eps > 0.0 ? eps : 0.0;
+    free(t);
+    return GRO_OK;
+}
+
 /* ------------------------------------------------------------------ whole solve
  * Steps 1-3 of the method for one decode position.  All per-support arrays are in
  * ratio order (position 0 = largest drf/tgt) and have k entries (psi: k+1).
  * method: 1 = proportional fitting alone, 2 = damped Newton (default).
+ * tau > 0 (Algorithm 1): each system is solved on its truncation set alone, to gradient norm 5 tau (`tol` is
+ * then not used); the weights of the tokens outside the sets are 0 (the guarantees of Thms "Inner / Outer
+ * Convex Solver" hold for any value there).  For an outer block the tuples counted are those inside
+ * (H* u T)^n, so its higher-ratio mass is drf(H*) plus the T-part of the higher outer blocks.
  */
 int gro_solve(const double *tl, const double *dl, int V, int n, int topk, double Tt, double Td,
-              int route, int method, double tol, int max_iter,
+              int route, int method, double tol, int max_iter, double tau,
               double *tgt_full, double *drf_full,
               int *k_out, int *order, double *tgt_pos, double *drf_pos, double *psi,
               int *jstar_out, double *alpha_star_out, double *p, double *r, int *block, int *nblocks_out,
@@ -480,6 +539,51 @@ int gro_solve(const double *tl, const double *dl, int V, int n, int topk, double
     *k_out = k; *jstar_out = jstar; *nblocks_out = nb;
 
     int status = GRO_OK, iters = 0; double gnorm = 0.0;
+    if (tau > 0.0) {
+        /* truncated variant: gather each system's T-part, solve it to 5 tau, scatter the weights back */
+        int *in_T = (int *)malloc(sizeof(int) * (size_t)(k > 0 ? k : 1));
+        int *map = (int *)malloc(sizeof(int) * (size_t)(k > 0 ? k : 1));
+        double *dT = (double *)malloc(sizeof(double) * (size_t)(3 * k + 3));
+        double *rT = dT + k + 1, *wT = rT + k + 1;
+        gro_truncation_sets(k, jstar, order, drf_pos, n, tau, in_T, NULL, NULL);
+        for (int j = 0; j < k; j++) w[j] = 0.0;
+        double stop = 5.0 * tau;
+        int m = 0;
+        for (int j = 0; j < jstar; j++) if (in_T[j]) { dT[m] = drf_pos[j]; rT[m] = tgt_pos[j]; map[m] = j; m++; }
+        if (m > 0) {
+            double gn = 0.0; int it = 0;
+            int st = (method == 1) ? gro_ipf(route, m, dT, rT, n, 0.0, 1, stop, max_iter, wT, &gn, &it)
+                                   : gro_newton(route, m, dT, rT, n, 0.0, 1, stop, max_iter, wT, &gn, &it);
+            if (st != GRO_OK) status = GRO_NOT_CONVERGED;
+            gnorm += gn; iters += it;
+            for (int q = 0; q < m; q++) w[map[q]] = wT[q];
+        }
+        double DH = 0.0;
+        for (int j = 0; j < jstar; j++) DH += drf_pos[j];
+        for (int b = nb - 1; b >= 0; b--) {         /* from the highest ratio down, the T-mass above accumulates */
+            int lo = -1, hi = -1;
+            for (int j = jstar; j < k; j++) if (block[j] == b) { if (lo < 0) lo = j; hi = j; }
+            if (lo < 0) continue;
+            double hT = DH;
+            for (int j = jstar; j < lo; j++) if (in_T[j]) hT += drf_pos[j];
+            m = 0;
+            for (int j = lo; j <= hi; j++) if (in_T[j]) { dT[m] = drf_pos[j]; rT[m] = p[j]; map[m] = j; m++; }
+            if (m == 1) w[map[0]] = 1.0;
+            if (m >= 2) {
+                double gn = 0.0; int it = 0;
+                int st = (method == 1) ? gro_ipf(route, m, dT, rT, n, hT, 0, stop, max_iter, wT, &gn, &it)
+                                       : gro_newton(route, m, dT, rT, n, hT, 0, stop, max_iter, wT, &gn, &it);
+                if (st != GRO_OK) status = GRO_NOT_CONVERGED;
+                gnorm += gn; iters += it;
+                for (int q = 0; q < m; q++) w[map[q]] = wT[q];
+            }
+        }
+        free(in_T); free(map); free(dT);
+        if (gnorm_out) *gnorm_out = gnorm;
+        if (iters_out) *iters_out = iters;
+        free(ids); free(Tg); free(Dr);
+        return status;
+    }
     /* inner system on H* (positions 0..jstar-1), rhs = tgt */
     {
         double gn = 0.0; int it = 0;
@@ -513,7 +617,8 @@ int gro_solve(const double *tl, const double *dl, int V, int n, int topk, double
  *   all of U in H*:  pi(i) = w_i / (1 + sum_U w),  rho = 1 / (1 + sum_U w) goes to
  *                    the resample distribution r / (1 - alpha*);
  *   otherwise:       B = lowest-ratio block met by U; pi(i) = w_i / sum_{U n B} w on
- *                    U n B, 0 on the rest of U, rho = 0.
+ *                    U n B, 0 on the rest of U, rho = 0.  (Truncated variant: when every
+ *                    token of U n B carries weight 0 they share the tuple equally.)
  * U_out / pi_out have up to n entries; returns |U| or a negative error.
  */
 int gro_slice(int k, int n, int jstar, const int *order, const int *block, const double *w,
@@ -539,8 +644,10 @@ int gro_slice(int k, int n, int jstar, const int *order, const int *block, const
     } else {
         int b = block[maxpos];
         double W = 0.0;
-        for (int u = 0; u < nu; u++) if (block[pos[u]] == b) W += w[pos[u]];
-        for (int u = 0; u < nu; u++) pi_out[u] = (block[pos[u]] == b) ? w[pos[u]] / W : 0.0;
+        int cnt = 0;
+        for (int u = 0; u < nu; u++) if (block[pos[u]] == b) { W += w[pos[u]]; cnt++; }
+        for (int u = 0; u < nu; u++)
+            pi_out[u] = (block[pos[u]] == b) ? (W > 0.0 ? w[pos[u]] / W : 1.0 / cnt) : 0.0;
         *rho_out = 0.0;
     }
     free(pos);
@@ -585,7 +692,7 @@ int gro_draw(int nu, const int *U, const double *pi, double rho, const double *r
  * pointers are not NULL -- the slice (U padded with -1, pi padded with 0, rho).
  */
 int gro_solve_verify_batch(const double *tl, const double *dl, int batch, int V, int n, int topk,
-                           double Tt, double Td, int route, int method, double tol, int max_iter,
+                           double Tt, double Td, int route, int method, double tol, int max_iter, double tau,
                            const int *draft_tokens, const float *uniforms,
                            double *alpha_star, int *token, int *accepted, int *status,
                            int *U_out, double *pi_out, double *rho_out, double *gnorm_out, int *iters_out,
@@ -607,7 +714,7 @@ int gro_solve_verify_batch(const double *tl, const double *dl, int batch, int V,
         double *tgt_pos = buf, *drf_pos = buf + k, *psi = buf + 2 * k, *p = buf + 3 * k + 1,
                *r = buf + 4 * k + 1, *w = buf + 5 * k + 1;
         int kk = 0, jstar = 0, nb = 0, iters = 0; double gn = 0.0, as = 0.0;
-        int st = gro_solve(tlb, dlb, V, n, topk, Tt, Td, route, method, tol, max_iter, tgt, drf, &kk, order,
+        int st = gro_solve(tlb, dlb, V, n, topk, Tt, Td, route, method, tol, max_iter, tau, tgt, drf, &kk, order,
                            tgt_pos, drf_pos, psi, &jstar, &as, p, r, block, &nb, w, &gn, &iters);
         alpha_star[b] = as;
         if (gnorm_out) gnorm_out[b] = gn;
@@ -723,6 +830,69 @@ int gro_certify_batch(const double *tl, const double *dl, int batch, int V, int 
         for (int j = 0; j <= kcap; j++) psi_out[(size_t)b * (kcap + 1) + j] = j <= kk ? psi[j] : 0.0;
         free(tgt); free(drf); free(ids); free(order); free(block); free(buf);
     }
+    return GRO_OK;
+}
+
+/* ------------------------------------------------------------------ marginals of a rule
+ * For ANY weights (zeros allowed, as the truncated variant leaves them) the rule of gro_slice defines a coupling;
+ * this returns what Lemma "Approximation Guarantee" bounds: the L1 distance of its emitted-token marginal from the
+ * target and its acceptance (= sum of the flows p'_i the tokens receive from the tuples that contain them).
+ * Flows by the integral route: the inner system on all of H* with the given weights; per outer block the
+ * tokens of positive weight (the block's zero-weight tokens take nothing from tuples that contain one of those,
+ * so their mass joins the higher-ratio mass), and the zero-weight tokens among themselves with equal weights.
+ * Emitted marginal (Eq. "approx-c"): p'_i on H*; p'_i + r_i rho / R on outer support tokens; tgt_i rho / R off the
+ * support, with rho = drf(H*)^n - sum_{H*} p'_j the mass left to the resample segment and R = 1 - alpha*.
+ * Arrays in ratio order, k entries; Dr = prefix sums of drf (k + 1 entries).
+ */
+int gro_rule_deviation(int k, int n, int jstar, int nblocks, const int *block, const double *tgt_pos,
+                       const double *drf_pos, const double *r, const double *w, double alpha_star,
+                       double *l1_out, double *accept_out, double *flow_out)
+{
+    double *flow = (double *)calloc((size_t)(k > 0 ? k : 1), sizeof(double));
+    double *dd = (double *)malloc(sizeof(double) * (size_t)(3 * k + 3));
+    double *ww = dd + k + 1, *gg = ww + k + 1;
+    int *map = (int *)malloc(sizeof(int) * (size_t)(k > 0 ? k : 1));
+    double DH = 0.0, tsup = 0.0;
+    for (int j = 0; j < jstar; j++) DH += drf_pos[j];
+    for (int j = 0; j < k; j++) tsup += tgt_pos[j];
+    if (jstar > 0) {
+        gro_grad_g2(jstar, drf_pos, w, n, 0.0, 1, gg);
+        for (int j = 0; j < jstar; j++) flow[j] = w[j] > 0.0 ? gg[j] : 0.0;
+    }
+    double above = DH;                 /* draft mass of everything of higher ratio than the current block */
+    for (int b = nblocks - 1; b >= 0; b--) {
+        int lo = -1, hi = -1;
+        for (int j = jstar; j < k; j++) if (block[j] == b) { if (lo < 0) lo = j; hi = j; }
+        if (lo < 0) continue;
+        double dz = 0.0;
+        int mp = 0, mz = 0;
+        for (int j = lo; j <= hi; j++) if (!(w[j] > 0.0)) dz += drf_pos[j];
+        for (int j = lo; j <= hi; j++) if (w[j] > 0.0) { dd[mp] = drf_pos[j]; ww[mp] = w[j]; map[mp] = j; mp++; }
+        if (mp > 0) {
+            gro_grad_g2(mp, dd, ww, n, above + dz, 0, gg);
+            for (int q = 0; q < mp; q++) flow[map[q]] = gg[q];
+        }
+        for (int j = lo; j <= hi; j++) if (!(w[j] > 0.0)) { dd[mz] = drf_pos[j]; ww[mz] = 1.0; map[mz] = j; mz++; }
+        if (mz > 0) {
+            gro_grad_g2(mz, dd, ww, n, above, 0, gg);
+            for (int q = 0; q < mz; q++) flow[map[q]] = gg[q];
+        }
+        for (int j = lo; j <= hi; j++) above += drf_pos[j];
+    }
+    double acc = 0.0, inner_flow = 0.0;
+    for (int j = 0; j < k; j++) acc += flow[j];
+    for (int j = 0; j < jstar; j++) inner_flow += flow[j];
+    double rho = pow(DH, (double)n) - inner_flow;
+    double R = 1.0 - alpha_star;
+    double share = R > 0.0 ? rho / R : 0.0;
+    double l1 = 0.0;
+    for (int j = 0; j < jstar; j++) l1 += fabs(flow[j] - tgt_pos[j]);
+    for (int j = jstar; j < k; j++) l1 += fabs(flow[j] + r[j] * share - tgt_pos[j]);
+    l1 += (1.0 - tsup) * fabs(share - 1.0);
+    if (l1_out) *l1_out = l1;
+    if (accept_out) *accept_out = acc;
+    if (flow_out) for (int j = 0; j < k; j++) flow_out[j] = flow[j];
+    free(flow); free(dd); free(map);
     return GRO_OK;
 }
 

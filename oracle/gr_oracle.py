@@ -130,7 +130,7 @@ class Solution:
 
 
 def solve(tl, dl, n, topk, Tt=1.0, Td=1.0, route=ROUTE_G2, tol=1e-12, max_iter=2000,
-          method=METHOD_NEWTON) -> Solution:
+          method=METHOD_NEWTON, tau=0.0) -> Solution:
     tl, dl = _f64(tl), _f64(dl)
     V = tl.shape[0]
     kmax = V if (topk <= 0 or topk >= V) else topk
@@ -142,7 +142,7 @@ def solve(tl, dl, n, topk, Tt=1.0, Td=1.0, route=ROUTE_G2, tol=1e-12, max_iter=2
     a = C.c_double(0); gn = C.c_double(0)
     D = C.c_double
     st = lib().gro_solve(_p(tl, D), _p(dl, D), V, int(n), int(topk), D(Tt), D(Td), int(route), int(method), D(tol), int(max_iter),
-                         _p(tgt, D), _p(drf, D), C.byref(k), _p(order, C.c_int), _p(tgt_pos, D), _p(drf_pos, D),
+                         D(tau), _p(tgt, D), _p(drf, D), C.byref(k), _p(order, C.c_int), _p(tgt_pos, D), _p(drf_pos, D),
                          _p(psi, D), C.byref(jstar), C.byref(a), _p(p, D), _p(r, D), _p(block, C.c_int),
                          C.byref(nb), _p(w, D), C.byref(gn), C.byref(it))
     if st < 0:
@@ -197,7 +197,7 @@ class BatchResult:
 
 
 def solve_verify_batch(tl, dl, n, topk, Tt, Td, draft_tokens, uniforms, route=ROUTE_G2, tol=1e-12,
-                       max_iter=2000, method=METHOD_NEWTON) -> BatchResult:
+                       max_iter=2000, method=METHOD_NEWTON, tau=0.0) -> BatchResult:
     tl, dl = _f64(tl), _f64(dl)
     B, V = tl.shape
     toks = _i32(draft_tokens); uni = np.ascontiguousarray(uniforms, dtype=np.float32)
@@ -211,7 +211,7 @@ def solve_verify_batch(tl, dl, n, topk, Tt, Td, draft_tokens, uniforms, route=RO
     w = np.zeros((B, kcap)); r = np.zeros((B, kcap)); p = np.zeros((B, kcap)); psi = np.zeros((B, kcap + 1))
     D = C.c_double
     lib().gro_solve_verify_batch(_p(tl, D), _p(dl, D), B, V, int(n), int(topk), D(Tt), D(Td), int(route), int(method), D(tol),
-                                 int(max_iter), _p(toks, C.c_int), _p(uni, C.c_float), _p(a, D), _p(token, C.c_int),
+                                 int(max_iter), D(tau), _p(toks, C.c_int), _p(uni, C.c_float), _p(a, D), _p(token, C.c_int),
                                  _p(acc, C.c_int), _p(status, C.c_int), _p(U, C.c_int), _p(pi, D), _p(rho, D),
                                  _p(gn, D), _p(it, C.c_int), _p(js, C.c_int),
                                  kcap, _p(kk, C.c_int), _p(nb, C.c_int), _p(order, C.c_int), _p(block, C.c_int),
@@ -278,6 +278,31 @@ def draw_sweep_batch(tl, dl, n, topk, Tt, Td, res: BatchResult, draft_tokens, un
                                _p(toks, C.c_int), _p(uni, C.c_float), R, _p(token, C.c_int), _p(acc, C.c_int),
                                _p(margin, D))
     return token, acc, margin
+
+
+def truncation_sets(order, drf_pos, jstar, n, tau):
+    """Minimal truncation sets (Sec. 6.2-6.3): (in_T [k] of 0/1 in ratio order, gamma_T, epsilon_T)."""
+    order = _i32(order); d = _f64(drf_pos)
+    k = d.shape[0]
+    in_T = np.zeros(k, dtype=np.int32)
+    gam = C.c_double(0); eps = C.c_double(0)
+    lib().gro_truncation_sets(k, int(jstar), _p(order, C.c_int), _p(d, C.c_double), int(n), C.c_double(tau),
+                              _p(in_T, C.c_int), C.byref(gam), C.byref(eps))
+    return in_T, gam.value, eps.value
+
+
+def rule_deviation(sol: Solution, w=None):
+    """(L1 distance of the emitted-token marginal from the target, acceptance, flows [k]) of the rule that the
+    structure of `sol` and the weights `w` (default: its own; zeros allowed) define."""
+    k = sol.k
+    w = _f64(sol.w[:k] if w is None else w)
+    l1 = C.c_double(0); acc = C.c_double(0)
+    flow = np.zeros(max(k, 1))
+    D = C.c_double
+    lib().gro_rule_deviation(k, int(sol.n), int(sol.jstar), int(sol.nblocks), _p(_i32(sol.block[:k]), C.c_int),
+                             _p(_f64(sol.tgt_pos[:k]), D), _p(_f64(sol.drf_pos[:k]), D), _p(_f64(sol.r[:k]), D),
+                             _p(w, D), D(sol.alpha_star), C.byref(l1), C.byref(acc), _p(flow, D))
+    return l1.value, acc.value, flow[:k]
 
 
 def num_threads() -> int:

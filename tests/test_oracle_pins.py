@@ -392,3 +392,104 @@ def test_alpha_star_only_agrees_with_the_full_solve_and_with_enumeration():
         assert a == sol.alpha_star and js == sol.jstar
         tgt, drf, _, _ = O.distributions(tl, dl, topk, 1.0, 1.0)
         assert abs(a - (1.0 + BF.all_subset_psi(tgt, drf, n).min())) < 1e-13
+
+
+# ---------------------------------------------------------------- truncated variant (Sec. 6.2-6.3, Algorithm 1)
+
+def test_truncation_sets_are_minimal_and_meet_their_bounds():
+    rng = np.random.default_rng(631)
+    for V, n, tau in [(9, 2, 0.05), (10, 3, 0.01), (8, 4, 0.2), (10, 2, 1e-4)]:
+        for _ in range(4):
+            tl = 1.5 * rng.standard_normal(V); dl = tl + 1.2 * rng.standard_normal(V)
+            sol = O.solve(tl, dl, n, 0, tol=1e-6, max_iter=20)
+            k, js = sol.k, sol.jstar
+            in_T, gam, eps = O.truncation_sets(sol.order, sol.drf_pos, js, n, tau)
+            d = sol.drf_pos
+            D = d[:js].sum()
+            Tin = [j for j in range(js) if in_T[j]]; Tout = [j for j in range(js, k) if in_T[j]]
+            assert abs(gam - (D ** n - d[Tin].sum() ** n)) < 1e-14 and gam <= tau
+            assert abs(eps - (1.0 - (D + d[Tout].sum()) ** n)) < 1e-14 and eps <= tau
+            # no smaller subset meets the bound (all subsets of one size less)
+            if Tin:
+                best = max(d[list(S)].sum() for S in itertools.combinations(range(js), len(Tin) - 1)) if len(Tin) > 1 else 0.0
+                assert D ** n - best ** n > tau
+            if Tout:
+                best = max(d[list(S)].sum() for S in itertools.combinations(range(js, k), len(Tout) - 1)) if len(Tout) > 1 else 0.0
+                assert 1.0 - (D + best) ** n > tau
+    # tau = 0 keeps every support token
+    in_T, gam, eps = O.truncation_sets(sol.order, sol.drf_pos, sol.jstar, n, 0.0)
+    assert in_T.all() and gam == 0.0 and eps == 0.0
+
+
+@pytest.mark.parametrize("V,n,topk", [(7, 2, 0), (8, 3, 0), (8, 2, 5), (6, 4, 0)])
+def test_truncated_rule_keeps_the_papers_guarantees(V, n, topk):
+    """The coupling assembled from the truncated solves (all tuples enumerated): within 15 tau of the target in L1,
+    acceptance within 10 tau of the optimum, column sums exact (Lemma "Approximation Guarantee", Sec. 6.3)."""
+    rng = np.random.default_rng(V * 1000 + n * 10 + topk)
+    used_truncation = 0
+    for tau in (0.1, 0.02, 1e-3):
+        for _ in range(3):
+            tl = 1.5 * rng.standard_normal(V); dl = tl + 1.0 * rng.standard_normal(V)
+            sol = O.solve(tl, dl, n, topk, tau=tau)
+            used_truncation += int(np.any(sol.w[: sol.k] == 0.0))
+            rowsum, acc = _coupling(sol, n)
+            assert np.abs(rowsum - sol.tgt_full).sum() <= 15 * tau
+            assert abs(acc - sol.alpha_star) <= 10 * tau
+            # the marginals computed without enumeration agree with the enumerated ones
+            l1, acc2, flow = O.rule_deviation(sol)
+            assert abs(l1 - np.abs(rowsum - sol.tgt_full).sum()) < 1e-11
+            assert abs(acc2 - acc) < 1e-11
+    assert used_truncation > 0
+
+
+def test_truncated_rule_tends_to_the_exact_one():
+    rng = np.random.default_rng(99)
+    tl = 1.5 * rng.standard_normal(12); dl = tl + 0.9 * rng.standard_normal(12)
+    exact = O.solve(tl, dl, 3, 0, tol=1e-13)
+    tiny = O.solve(tl, dl, 3, 0, tau=1e-14)
+    assert np.all(tiny.w[: tiny.k] > 0)
+    assert np.allclose(tiny.w, exact.w, rtol=1e-6)
+    devs = [O.rule_deviation(O.solve(tl, dl, 3, 0, tau=t))[0] for t in (0.1, 1e-2, 1e-3, 1e-5)]
+    assert devs[-1] < 1e-4 and devs[-1] <= devs[0] + 1e-12
+
+
+def test_rule_marginals_for_arbitrary_weights_match_enumeration():
+    """gro_rule_deviation against the enumerated coupling for weights that solve nothing, zeros included
+    (whole blocks of zeros share their tuples equally)."""
+    rng = np.random.default_rng(5150)
+    seen_zero_block = 0
+    for V, n, topk in [(7, 3, 0), (8, 2, 0), (7, 2, 5)]:
+        for _ in range(4):
+            tl = 1.5 * rng.standard_normal(V); dl = tl + 1.3 * rng.standard_normal(V)
+            sol = O.solve(tl, dl, n, topk, tol=1e-6, max_iter=30)
+            w = np.exp(rng.normal(0, 1.5, sol.k))
+            w[rng.random(sol.k) < 0.4] = 0.0
+            for b in range(sol.nblocks):
+                if rng.random() < 0.3:
+                    w[sol.block[: sol.k] == b] = 0.0
+                    seen_zero_block += 1
+            sol2 = O.Solution(**{**sol.__dict__, "w": w})
+            rowsum, acc = _coupling(sol2, n)
+            l1, acc2, flow = O.rule_deviation(sol, w)
+            assert abs(acc2 - acc) < 1e-11
+            assert abs(l1 - np.abs(rowsum - sol.tgt_full).sum()) < 1e-11
+    assert seen_zero_block > 0
+
+
+def test_certificate_and_draw_sweep_helpers():
+    """The batch helpers used by the GPU tests: the certificate vanishes at the oracle's own weights and does not at
+    perturbed ones; the sweep's first draw is the batch driver's draw."""
+    wl = W.config1(batch=6)
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    tk = wl.draft_tokens.numpy(); un = wl.uniforms.numpy()
+    res = O.solve_verify_batch(tl, dl, wl.n, wl.topk, 1.0, 1.0, tk, un)
+    cert = O.certify_batch(tl, dl, wl.n, wl.topk, 1.0, 1.0, res.w, lse=None)
+    assert cert.gnorm.max() < 1e-11 and np.array_equal(cert.order, res.order) and np.array_equal(cert.block, res.block)
+    bad = O.certify_batch(tl, dl, wl.n, wl.topk, 1.0, 1.0, res.w * (1.0 + 0.01 * (np.arange(res.w.shape[1]) % 3)))
+    solved = [b for b in range(6) if res.jstar[b] >= 2 or np.any(np.bincount(res.block[b][res.block[b] >= 0]) >= 2)]
+    assert all(bad.gnorm[b] > 1e-6 for b in solved) and len(solved) >= 3
+    # a log-sum-exp given from outside: off by delta, the certificate against the shifted target sees ~delta
+    shifted = O.certify_batch(tl, dl, wl.n, wl.topk, 1.0, 1.0, res.w, lse=cert.lse_target + 1e-6)
+    assert np.all(shifted.gnorm_lse[solved] > 1e-8) and shifted.gnorm.max() < 1e-11
+    tok, acc, margin = O.draw_sweep_batch(tl, dl, wl.n, wl.topk, 1.0, 1.0, res, tk, un[:, None, :])
+    assert np.array_equal(tok[:, 0], res.token) and np.array_equal(acc[:, 0], res.accepted) and np.all(margin >= 0)
