@@ -77,6 +77,15 @@ extern "C" {
  *   force_robust  non-zero sends every shape to the general (slower) solve kernel;
  *              by default supports of at most 128 tokens with n <= 16 take a faster
  *              kernel that computes the same rule.                  default 0
+ *   tau        error threshold of Algorithm 1 (Sec. 6.2 "tunable errors", Sec. 6.3).  0 solves the
+ *              convex programs on the whole support (the default: both tunable errors are 0 and `tol`
+ *              is the stopping rule).  tau in (0, 1] selects the truncated variant: the inner system
+ *              is solved on the fewest tokens T of H* with gamma_T = drf(H*)^n - drf(T)^n <= tau, every
+ *              outer block on the fewest outer tokens T with epsilon_T = 1 - (drf(H*) + drf(T))^n <= tau
+ *              (largest drf first), each to gradient norm 5 tau (`tol` is then not used); tokens outside
+ *              the sets keep weight 0 (a tuple served only by such tokens of an outer block is shared
+ *              equally among them).  The emitted token then follows the target within 15 tau in L1 and
+ *              the acceptance is within 10 tau of alpha* (Lemma "Approximation Guarantee").     default 0
  */
 typedef struct gr_options {
     double tol;
@@ -84,6 +93,7 @@ typedef struct gr_options {
     double quad_step;
     void*  scan_done_event;
     int    force_robust;
+    double tau;
 } gr_options;
 
 /*

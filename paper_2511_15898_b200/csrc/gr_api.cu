@@ -6,15 +6,15 @@ namespace gr {
 // The fast kernel covers supports up to 128 tokens with n <= 16; everything else, and any instance the fast
 // kernel could not finish, takes the robust kernel.
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                     double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
+                     double temp_d, double tol, int max_iters, double qstep, double tau, int batch, int force_robust,
                      float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st)
 {
     int rc = force_robust ? 1
                           : launch_fast(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep,
-                                        batch, alpha_out, status_out, fa, st);
+                                        tau, batch, alpha_out, status_out, fa, st);
     if (rc < 0) return rc;
     // rc == 1: no fast variant, the robust kernel does everything; rc == 0: it redoes what the fast one flagged
-    return launch_solve(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch,
+    return launch_solve(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, tau, batch,
                         rc == 0 ? 1 : 0, alpha_out, status_out, fa, st);
 }
 
@@ -30,13 +30,14 @@ int check_solve_args(const void* q_logits, const void* p_logits, int dtype, int 
     if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
     if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
         return GR_E_INVALID;
-    out->tol = 1e-9; out->qstep = 0.4; out->max_iters = 40;
+    out->tol = 1e-9; out->qstep = 0.4; out->max_iters = 40; out->tau = 0.0;
     out->scan_done = nullptr; out->force_robust = 0;
     if (opt) {
         out->scan_done = (cudaEvent_t)opt->scan_done_event;
         out->force_robust = opt->force_robust;
-        out->tol = opt->tol; out->max_iters = opt->max_iters; out->qstep = opt->quad_step;
+        out->tol = opt->tol; out->max_iters = opt->max_iters; out->qstep = opt->quad_step; out->tau = opt->tau;
         if (!(out->tol > 0.0) || out->max_iters < 1 || !(out->qstep >= 0.05 && out->qstep <= 2.0)) return GR_E_INVALID;
+        if (!(out->tau >= 0.0) || !(out->tau <= 1.0)) return GR_E_INVALID;
     }
     out->kfull = (topk <= 0 || topk >= V) ? V : topk;
     out->kcap = kcap_of(V, topk);
@@ -79,7 +80,7 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
     if (batch == 0) return GR_OK;
     if (!workspace) return GR_E_NULL;
     if ((uintptr_t)workspace & 15) return GR_E_ALIGN;
-    const double tol = su.tol, qstep = su.qstep;
+    const double tol = su.tol, qstep = su.qstep, tau = su.tau;
     const int max_iters = su.max_iters, force_robust = su.force_robust;
     cudaEvent_t scan_done = su.scan_done;
     const int kfull = su.kfull, kcap = su.kcap, pstride = su.pstride;
@@ -90,8 +91,8 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     int rc = gr::launch_solve_any((const char*)workspace, (char*)params, pstride, kcap, V, n, topk,
-                                  (double)temp_target, (double)temp_draft, tol, max_iters, qstep, batch, force_robust,
-                                  alpha_star, status, fa, st);
+                                  (double)temp_target, (double)temp_draft, tol, max_iters, qstep, tau, batch,
+                                  force_robust, alpha_star, status, fa, st);
     if (rc != GR_OK) return rc;
     if (full_large) {
         // no rule is solved for this shape, but the optimal acceptance still is (sort + prefix scan)

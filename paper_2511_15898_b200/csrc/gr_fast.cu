@@ -6,8 +6,8 @@ namespace gr {
 
 #define GR_FAST_ARGS                                                                                              \
     const char *ws, char *params, int pstride, int kcap, int V, int n, int topk, double temp_t, double temp_d,   \
-        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, FusedArgs fa,     \
-        cudaStream_t st
+        double tol, int max_iters, double qstep, double tau, int batch, float *alpha_out, int *status_out,       \
+        FusedArgs fa, cudaStream_t st
 namespace fast64 {
 int launch_fast_n4(GR_FAST_ARGS);
 int launch_fast_n8(GR_FAST_ARGS);
@@ -23,7 +23,7 @@ int launch_fast_n16(GR_FAST_ARGS);
 int launch_fast(GR_FAST_ARGS)
 {
     if (kcap <= 0 || kcap > 128 || n > 16 || n < 2) return 1;
-#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, fa, st
+#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, tau, batch, alpha_out, status_out, fa, st
     if (kcap <= 64) {
         if (n <= 4) return fast64::launch_fast_n4(GR_FAST_PASS);
         if (n <= 8) return fast64::launch_fast_n8(GR_FAST_PASS);

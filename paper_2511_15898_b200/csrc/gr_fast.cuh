@@ -71,7 +71,7 @@ struct FastLayout {
         jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
         o += (kMP * (kMP + 1) + 1) / 2;
         ints = o * 8;
-        total_bytes = ints + KP * 3 * 4 + 64;
+        total_bytes = ints + KP * 4 * 4 + 64;
     }
 };
 static inline int fast_smem_bytes(int KP, int NT) { return FastLayout(KP, NT).total_bytes; }
@@ -80,7 +80,7 @@ struct FSm {
     double *d, *tg, *p, *r, *key, *psi, *Dr, *alpha, *alpha_prev, *delta, *w, *g, *g2, *col, *gw, *g2w, *tq, *cq,
         *scal, *J;
     float *AS, *HS, *Jacc;
-    int *id, *blk, *itmp;
+    int *id, *blk, *itmp, *trunc;
     int KP;
 };
 enum { SC_Q = 0, SC_FAIL = 1, SC_RED = 8 };
@@ -814,7 +814,7 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
 template <int NT, int TPL>
 __global__ void __launch_bounds__(kFT, kFCtas)
 fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
-                  double temp_t, double temp_d, double tol, int max_iters, double qstep,
+                  double temp_t, double temp_d, double tol, int max_iters, double qstep, double tau,
                   float* __restrict__ alpha_out, int* __restrict__ status_out, FusedArgs fa)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -846,7 +846,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     sm.HS = sm.AS + kJC * NT * kMS;
     sm.Jacc = reinterpret_cast<float*>(smem_raw + L.jacc_bytes_off);
     int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
-    sm.id = ib; sm.blk = ib + KP; sm.itmp = ib + 2 * KP;
+    sm.id = ib; sm.blk = ib + KP; sm.itmp = ib + 2 * KP; sm.trunc = ib + 3 * KP;
     sm.KP = KP;
     PrepSm ps;
     ps.d = sm.d; ps.tg = sm.tg; ps.p = sm.p; ps.r = sm.r; ps.key = sm.key; ps.psi = sm.psi; ps.Dr = sm.Dr;
@@ -856,17 +856,35 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
 
     int status = GR_OK, iters_total = 0;
     double gnorm_total = 0.0;
-    if (tid < k) pv.w[tid] = 1.0;
+    // Truncated variant (Algorithm 1 with an error threshold): every system is solved on its truncation set alone,
+    // to gradient norm 5 tau; the other tokens keep weight 0.  The gathered arrays reuse what the preparation no
+    // longer needs.
+    const bool trunc = tau > 0.0;
+    if (trunc) {
+        truncation_sets(ps, sm.trunc, sm.itmp, k, jstar, n, tau);
+        tol = 5.0 * tau;
+    }
+    double* dT = sm.key; double* rT = sm.psi; int* tmap = sm.itmp;
+    if (tid < k) pv.w[tid] = trunc ? 0.0 : 1.0;
     // with the drafted tuple at hand only the system it selects is solved
     const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
     bool skipped = false;
     if (jstar > 0 && sel >= 0) skipped = true;
     if (jstar > 0 && sel < 0) {
-        double gn; int it;
-        const int st = fast_system<NT, TPL>(sm, jstar, n, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
-        if (st != GR_OK) status = kNeedFallback;
+        double gn = 0.0; int it = 0;
+        if (!trunc) {
+            const int st = fast_system<NT, TPL>(sm, jstar, n, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+            if (st != GR_OK) status = kNeedFallback;
+            if (tid < jstar) pv.w[tid] = sm.w[tid];
+        } else {
+            const int mT = gather_truncated(sm.trunc, 0, jstar, sm.d, sm.tg, dT, rT, tmap, &s_sel);
+            if (mT > 0) {
+                const int st = fast_system<NT, TPL>(sm, mT, n, dT, rT, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+                if (st != GR_OK) status = kNeedFallback;
+                if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
+            }
+        }
         gnorm_total += gn; iters_total += it;
-        if (tid < jstar) pv.w[tid] = sm.w[tid];
         __syncthreads();
     }
     int lo = jstar;
@@ -875,14 +893,33 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
         const int bk = sm.blk[lo];
         while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
         const int m = hi - lo + 1;
-        if (m >= 2 && sel != -2 && sel != bk) skipped = true;
-        if (m >= 2 && (sel == -2 || sel == bk)) {
-            double gn; int it;
-            const int st = fast_system<NT, TPL>(sm, m, n, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep,
-                                                &gn, &it);
-            if (st != GR_OK) status = kNeedFallback;
-            gnorm_total += gn; iters_total += it;
-            if (tid < m) pv.w[lo + tid] = sm.w[tid];
+        const bool wanted = sel == -2 || sel == bk;
+        if (!trunc) {
+            if (m >= 2 && !wanted) skipped = true;
+            if (m >= 2 && wanted) {
+                double gn; int it;
+                const int st = fast_system<NT, TPL>(sm, m, n, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep,
+                                                    &gn, &it);
+                if (st != GR_OK) status = kNeedFallback;
+                gnorm_total += gn; iters_total += it;
+                if (tid < m) pv.w[lo + tid] = sm.w[tid];
+                __syncthreads();
+            }
+        } else {
+            // tuples counted: those inside (H* u T)^n, so the mass above the block is drf(H*) plus the T-part of the
+            // higher-ratio outer blocks
+            double hT = sm.Dr[jstar];
+            for (int j = jstar; j < lo; j++) hT += sm.trunc[j] ? sm.d[j] : 0.0;
+            const int mT = gather_truncated(sm.trunc, lo, hi + 1, sm.d, sm.p, dT, rT, tmap, &s_sel);
+            if (mT == 1 && tid == 0) pv.w[tmap[0]] = 1.0;
+            if (mT >= 2 && !wanted) skipped = true;
+            if (mT >= 2 && wanted) {
+                double gn; int it;
+                const int st = fast_system<NT, TPL>(sm, mT, n, dT, rT, hT, 0, tol, max_iters, qstep, &gn, &it);
+                if (st != GR_OK) status = kNeedFallback;
+                gnorm_total += gn; iters_total += it;
+                if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
+            }
             __syncthreads();
         }
         lo = hi + 1;
@@ -897,7 +934,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
 
 template <int NT, int TPL>
 int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                         double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out,
+                         double temp_d, double tol, int max_iters, double qstep, double tau, int batch, float* alpha_out,
                          int* status_out, FusedArgs fa, cudaStream_t st)
 {
     const int smem = fast_smem_bytes(kcap, NT);
@@ -916,16 +953,16 @@ int launch_fast_t(const char* ws, char* params, int pstride, int kcap, int V, in
         configured[dev] = true;
     }
     fast_solve_kernel<NT, TPL><<<batch, kFT, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
-                                                         max_iters, qstep, alpha_out, status_out, fa);
+                                                         max_iters, qstep, tau, alpha_out, status_out, fa);
     return GR_OK;
 }
 
 // One translation unit per series length instantiates its kernels (they compile in parallel).
 #define GR_FAST_ARGS                                                                                              \
     const char *ws, char *params, int pstride, int kcap, int V, int n, int topk, double temp_t, double temp_d,   \
-        double tol, int max_iters, double qstep, int batch, float *alpha_out, int *status_out, FusedArgs fa,     \
-        cudaStream_t st
-#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, batch, alpha_out, status_out, fa, st
+        double tol, int max_iters, double qstep, double tau, int batch, float *alpha_out, int *status_out,       \
+        FusedArgs fa, cudaStream_t st
+#define GR_FAST_PASS ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol, max_iters, qstep, tau, batch, alpha_out, status_out, fa, st
 #define GR_FAST_INSTANTIATE(NT)                                                                \
     int launch_fast_n##NT(GR_FAST_ARGS) {                                                       \
         return kcap <= 32 * (kRL - 1) ? launch_fast_t<NT, kRL - 1>(GR_FAST_PASS)                    \

@@ -8,13 +8,13 @@ namespace gr {
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
-                 int* status_out, FusedArgs fa, cudaStream_t st);
+                 double temp_d, double tol, int max_iters, double qstep, double tau, int batch, int only_flagged,
+                 float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st);
 int launch_fast(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                double temp_d, double tol, int max_iters, double qstep, int batch, float* alpha_out, int* status_out,
-                FusedArgs fa, cudaStream_t st);
+                double temp_d, double tol, int max_iters, double qstep, double tau, int batch, float* alpha_out,
+                int* status_out, FusedArgs fa, cudaStream_t st);
 int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                     double temp_d, double tol, int max_iters, double qstep, int batch, int force_robust,
+                     double temp_d, double tol, int max_iters, double qstep, double tau, int batch, int force_robust,
                      float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st);
 size_t fullsort_scratch_bytes(int V);
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
@@ -30,7 +30,7 @@ void launch_read_rule(const char* params, int batch, int kcap, int* ids, int* bl
 
 // The solver options after defaults and range checks.
 struct SolveSetup {
-    double tol, qstep;
+    double tol, qstep, tau;
     int max_iters, force_robust;
     cudaEvent_t scan_done;
     int kfull, kcap, pstride;      // support size asked for, capacity of the per-support arrays (0: beyond it), params stride

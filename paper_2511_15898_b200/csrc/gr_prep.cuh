@@ -178,6 +178,67 @@ __device__ inline PrepResult prep_instance(const PrepSm& sm, const WsView& wv, H
     return pr;
 }
 
+// Truncation sets of the truncated variant (Sec. 6.2 "tunable errors", Sec. 6.3, Algorithm 1): the fewest tokens with
+//   inner:  T in H*,       gamma_T   = drf(H*)^n - drf(T)^n      <= tau,
+//   outer:  T in V \ H*,   epsilon_T = 1 - (drf(H*) + drf(T))^n  <= tau,
+// i.e. tokens in decreasing drf (equal drf: smaller id first) until the bound holds.  in_T[pos] = 1 / 0 for the
+// k support positions (ratio order); scratch: k ints.  Every thread of the CTA calls it (blockDim.x >= k).
+__device__ inline void truncation_sets(const PrepSm& sm, int* in_T, int* scratch, int k, int jstar, int n, double tau)
+{
+    const int tid = threadIdx.x;
+    if (tid < k) {
+        // rank inside the own group (H* or the outer support) by (drf descending, id ascending)
+        const bool inner = tid < jstar;
+        const int lo = inner ? 0 : jstar, hi = inner ? jstar : k;
+        const double dv = sm.d[tid];
+        const int iv = sm.id[tid];
+        int rank = 0;
+        for (int j = lo; j < hi; j++) {
+            const double dj = sm.d[j];
+            rank += (dj > dv || (dj == dv && sm.id[j] < iv)) ? 1 : 0;
+        }
+        scratch[lo + rank] = tid;          // position of the group's rank-th token
+        in_T[tid] = 0;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        double D = 0.0;
+        for (int j = 0; j < jstar; j++) D += sm.d[j];
+        auto powi = [](double x, int e) { double r = 1.0; while (e > 0) { if (e & 1) r *= x; x *= x; e >>= 1; } return r; };
+        const double Dn = powi(D, n);
+        double c = 0.0, gam = Dn;
+        for (int q = 0; q < jstar && gam > tau; q++) {
+            const int pos = scratch[q];
+            c += sm.d[pos]; in_T[pos] = 1;
+            gam = Dn - powi(c, n);
+        }
+        c = D;
+        double eps = 1.0 - Dn;
+        for (int q = jstar; q < k && eps > tau; q++) {
+            const int pos = scratch[q];
+            c += sm.d[pos]; in_T[pos] = 1;
+            eps = 1.0 - powi(c, n);
+        }
+    }
+    __syncthreads();
+}
+
+// The T-part of positions lo .. hi-1 gathered into contiguous arrays (draft masses, right-hand sides, positions);
+// returns how many.  Every thread of the CTA calls it; `count` is one int of shared memory.
+__device__ inline int gather_truncated(const int* in_T, int lo, int hi, const double* d, const double* rhs, double* dT,
+                                       double* rT, int* map, int* count)
+{
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int m = 0;
+        for (int j = lo; j < hi; j++)
+            if (in_T[j]) { dT[m] = d[j]; rT[m] = rhs[j]; map[m] = j; m++; }
+        *count = m;
+    }
+    __syncthreads();
+    return *count;
+}
+
 // Rule arrays (except w, which the solvers write as they go) and the header.
 __device__ inline void write_rule(const PrepSm& sm, const ParamView& pv, int KP, const PrepResult& pr, int n,
                                   int status, double gnorm, int iters, float* alpha_out, int* status_out, long long b)

@@ -444,7 +444,7 @@ __device__ int solve_system(const Sm& sm, int m, const double* d, const double* 
 
 __global__ void __launch_bounds__(kSolveThreads)
 solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride, int kcap, int V, int n, int topk,
-             double temp_t, double temp_d, double tol, int max_iters, double qstep, int Qt, int only_flagged,
+             double temp_t, double temp_d, double tol, int max_iters, double qstep, double tau, int Qt, int only_flagged,
              float* __restrict__ alpha_out, int* __restrict__ status_out, FusedArgs fa)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -492,17 +492,35 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     // ---- convex minimisation: inner system on H*, then every outer block with two or more tokens
     int status = GR_OK, iters_total = 0;
     double gnorm_total = 0.0;
-    if (tid < k) pv.w[tid] = 1.0;
+    // Truncated variant (Algorithm 1 with an error threshold): every system is solved on its truncation set alone,
+    // to gradient norm 5 tau; the other tokens keep weight 0.  The gathered arrays reuse what the preparation no
+    // longer needs.
+    const bool trunc = tau > 0.0;
+    if (trunc) {
+        truncation_sets(ps, sm.order, sm.itmp, k, jstar, n, tau);
+        tol = 5.0 * tau;
+    }
+    double* dT = sm.key; double* rT = sm.psi; int* tmap = sm.itmp;
+    if (tid < k) pv.w[tid] = trunc ? 0.0 : 1.0;
     // with the drafted tuple at hand only the system it selects is solved
     const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
     bool skipped = false;
     if (jstar > 0 && sel >= 0) skipped = true;
     if (jstar > 0 && sel < 0) {
-        double gn; int it;
-        int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
-        if (st != GR_OK) status = GR_NOT_CONVERGED;
+        double gn = 0.0; int it = 0;
+        if (!trunc) {
+            int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+            if (st != GR_OK) status = GR_NOT_CONVERGED;
+            if (tid < jstar) pv.w[tid] = sm.w[tid];
+        } else {
+            const int mT = gather_truncated(sm.order, 0, jstar, sm.d, sm.tg, dT, rT, tmap, &s_sel);
+            if (mT > 0) {
+                int st = solve_system(sm, mT, dT, rT, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+                if (st != GR_OK) status = GR_NOT_CONVERGED;
+                if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
+            }
+        }
         gnorm_total += gn; iters_total += it;
-        if (tid < jstar) pv.w[tid] = sm.w[tid];
         __syncthreads();
     }
     {
@@ -512,13 +530,32 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
             const int bk = sm.blk[lo];
             while (hi + 1 < k && sm.blk[hi + 1] == bk) hi++;
             const int m = hi - lo + 1;
-            if (m >= 2 && sel != -2 && sel != bk) skipped = true;
-            if (m >= 2 && (sel == -2 || sel == bk)) {
-                double gn; int it;
-                int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it);
-                if (st != GR_OK) status = GR_NOT_CONVERGED;
-                gnorm_total += gn; iters_total += it;
-                if (tid < m) pv.w[lo + tid] = sm.w[tid];
+            const bool wanted = sel == -2 || sel == bk;
+            if (!trunc) {
+                if (m >= 2 && !wanted) skipped = true;
+                if (m >= 2 && wanted) {
+                    double gn; int it;
+                    int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it);
+                    if (st != GR_OK) status = GR_NOT_CONVERGED;
+                    gnorm_total += gn; iters_total += it;
+                    if (tid < m) pv.w[lo + tid] = sm.w[tid];
+                    __syncthreads();
+                }
+            } else {
+                // tuples counted: those inside (H* u T)^n, so the mass above the block is drf(H*) plus the T-part of
+                // the higher-ratio outer blocks
+                double hT = sm.Dr[jstar];
+                for (int j = jstar; j < lo; j++) hT += sm.order[j] ? sm.d[j] : 0.0;
+                const int mT = gather_truncated(sm.order, lo, hi + 1, sm.d, sm.p, dT, rT, tmap, &s_sel);
+                if (mT == 1 && tid == 0) pv.w[tmap[0]] = 1.0;
+                if (mT >= 2 && !wanted) skipped = true;
+                if (mT >= 2 && wanted) {
+                    double gn; int it;
+                    int st = solve_system(sm, mT, dT, rT, hT, 0, tol, max_iters, qstep, &gn, &it);
+                    if (st != GR_OK) status = GR_NOT_CONVERGED;
+                    gnorm_total += gn; iters_total += it;
+                    if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
+                }
                 __syncthreads();
             }
             lo = hi + 1;
@@ -534,8 +571,8 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
 }
 
 int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int n, int topk, double temp_t,
-                 double temp_d, double tol, int max_iters, double qstep, int batch, int only_flagged, float* alpha_out,
-                 int* status_out, FusedArgs fa, cudaStream_t st)
+                 double temp_d, double tol, int max_iters, double qstep, double tau, int batch, int only_flagged,
+                 float* alpha_out, int* status_out, FusedArgs fa, cudaStream_t st)
 {
     int Qt = 1, smem = 0;
     if (kcap > 0) {
@@ -556,7 +593,7 @@ int launch_solve(const char* ws, char* params, int pstride, int kcap, int V, int
         configured[dev] = true;
     }
     solve_kernel<<<batch, kSolveThreads, smem, st>>>(ws, params, pstride, kcap, V, n, topk, temp_t, temp_d, tol,
-                                                     max_iters, qstep, Qt, only_flagged, alpha_out, status_out, fa);
+                                                     max_iters, qstep, tau, Qt, only_flagged, alpha_out, status_out, fa);
     return GR_OK;
 }
 

@@ -41,7 +41,7 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     if (chk != GR_OK) return chk;
     if (batch > GR_STATIC_MAX_BATCH) return GR_E_TOO_LARGE;      // the built-in scratch holds this many instances
     if (batch == 0) return GR_OK;
-    const double tol = su.tol, qstep = su.qstep;
+    const double tol = su.tol, qstep = su.qstep, tau = su.tau;
     const int max_iters = su.max_iters, force_robust = su.force_robust;
     cudaEvent_t scan_done = su.scan_done;
     const int kfull = su.kfull, kcap = su.kcap;
@@ -58,7 +58,7 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     const int rc = gr::launch_solve_any(ws, (char*)params, pstride, kcap, V, n, topk, (double)temp_target,
-                                        (double)temp_draft, tol, max_iters, qstep, batch, force_robust, alpha_star,
+                                        (double)temp_draft, tol, max_iters, qstep, tau, batch, force_robust, alpha_star,
                                         status, gr::FusedArgs{nullptr, nullptr, nullptr, nullptr, nullptr}, st);
     if (rc != GR_OK) return rc;
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }

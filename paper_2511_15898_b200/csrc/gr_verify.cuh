@@ -172,7 +172,14 @@ __device__ inline int slice_instance(const Header* h, const ParamView& pv, int t
     }
     const double W = warp_sum(wv) + (inner ? 1.0 : 0.0);
     sl.uniq = uniq; sl.inner = inner;
-    sl.pi = wv / W;
+    if (W > 0.0) {
+        sl.pi = wv / W;
+    } else {
+        // (truncated variant) every served token carries weight 0: they share the tuple equally
+        const bool served = uniq && pv.blk[pos] == pv.blk[maxpos];
+        const int cnt = __popc(__ballot_sync(0xffffffffu, served));
+        sl.pi = served ? 1.0 / (double)cnt : 0.0;
+    }
     sl.rho = inner ? 1.0 / W : 0.0;
     return GR_OK;
 }

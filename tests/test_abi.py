@@ -67,12 +67,17 @@ def test_argument_errors_are_reported_before_any_launch(lib):
     assert call(opt=G.Options(tol=0.0)) == -1
     assert call(opt=G.Options(quad_step=5.0)) == -1
     assert call(opt=G.Options(max_iters=0)) == -1
+    assert call(opt=G.Options(tau=-1e-3)) == -1 and call(opt=G.Options(tau=1.5)) == -1
+    assert call(opt=G.Options(tau=float("nan"))) == -1
     assert call(V=100000, topk=500) == -5        # truncated support beyond GR_MAX_SUPPORT
     assert call(batch=0) == 0                    # an empty batch is a no-op
     assert G.gr_verify(0, A, A, 2, A, A, A, 0) == -2
     assert G.gr_verify(A, A, A, -1, A, A, A, 0) == -1
     assert G.gr_verify(A, A, A, 0, A, A, A, 0) == 0
     assert G.gr_read_rule(0, 1, 8, 0, 0, 0, 0, 0, 0, 0) == -2
+    assert G.gr_read_slice(0, A, 2, 4, A, A, A, A, 0) == -2 and G.gr_read_slice(A, A, 2, 4, 0, A, A, A, 0) == -2
+    assert G.gr_read_slice(A, A, 2, 0, A, A, A, A, 0) == -1 and G.gr_read_slice(A, A, -1, 4, A, A, A, A, 0) == -1
+    assert G.gr_read_slice(A + 4, A, 2, 4, A, A, A, A, 0) == -3 and G.gr_read_slice(A, A, 0, 4, A, A, A, A, 0) == 0
     # the fused entry: gr_solve's checks plus its own pointers
     def fused(**kw):
         a = dict(ok); a.update(kw)
