@@ -26,13 +26,30 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "solve+verify instances/sec at V=128256,n=8,top-k=50"
 UNIT = "instances/s"
 HEADLINE = dict(V=128256, n=8, topk=50, batch=1024, temp_target=0.7, temp_draft=1.0)
-BYTES_PER_INSTANCE = HEADLINE["V"] * (4 + 4)       # both fp32 logit rows, read once
-# dram__bytes_read + dram__bytes_write of scan_kernel per instance, from the ncu capture at batch 296
-# (profiles/scan_kernel_config3_batch296.md); traffic is proportional to the rows read
-SCAN_TRAFFIC_PER_INSTANCE = (305.128704e6 + 4.365568e6) / 296
+METRIC = "solve+verify instances/sec at V=128256,n=8,top-k=50"
+# DRAM bytes the streaming kernel moves per algorithmic byte (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture of scan_kernel on the headline shape at 296 instances, over the bytes of both logit rows; the
+# traffic of a launch is proportional to the rows it reads)
+SCAN_TRAFFIC_RATIO = 1.019
+DEFAULT_BATCH = {1: 64, 2: 256, 3: 1024, 4: 512, 5: 4096}
+ORACLE_SAMPLE = {1: 64, 2: 128, 3: 128, 4: 32, 5: 32}
+
+
+def make_workload(W, config, cell, batch, device, seed_offset=0):
+    """The benchmark configuration `config` (1..5) as a seeded synthetic workload; `cell` = (n, topk, sigma) picks
+    the cell of configuration 4's sweep (topk 0 = whole vocabulary)."""
+    if config == 1:
+        return W.config1(batch=batch, device=device, seed=1000 + seed_offset)
+    if config == 2:
+        return W.config2(batch=batch, device=device, seed=2000 + seed_offset)
+    if config == 3:
+        return W.config3(batch=batch, device=device, seed=3000 + seed_offset)
+    if config == 4:
+        n, topk, sigma = cell
+        return W.config4(int(n), int(topk), float(sigma), batch=batch, device=device)
+    return W.config5(batch=batch, device=device, seed=5000 + seed_offset, rows_per_pass=256)
 
 
 def _peaks():
@@ -105,24 +122,38 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = 16
-    wl = W.config3(batch=sample, device="cpu", seed=3000)
+    cfg = args.config
+    sample = {1: 16, 2: 16, 3: 16, 4: 8, 5: 4}[cfg]
+    wl = make_workload(W, cfg, args.cell, sample, "cpu")
+    kfull = wl.V if (wl.topk <= 0 or wl.topk >= wl.V) else wl.topk
     tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
     tk = wl.draft_tokens.numpy(); un = wl.uniforms.numpy()
+    metric = (METRIC if cfg == 3 else
+              f"solve+verify instances/sec at V={wl.V},n={wl.n},top-k={wl.topk if wl.topk else 'V'}")
+
+    def one_step():
+        if kfull > 4096:
+            # no convex solve is feasible on a support this large: the oracle's part is the optimal acceptance
+            for i in range(sample):
+                O.alpha_star_only(tl[i], dl[i], wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+        else:
+            O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, tk, un)
+
     for _ in range(max(args.warmup, 0)):
-        O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, tk, un)
+        one_step()
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, tk, un)
+        one_step()
     dt = time.perf_counter() - t0
     val = sample * args.steps / dt
     cores = O.num_threads()
     out = {
-        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "impl": "reference", "metric": metric, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(args.steps, 1), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "config3: V=128256 n=8 top-k=50 fp32 logits, target temp 0.7, draft temp 1.0",
-                   "sample": f"{sample} instances per step (of the 1024-instance batch)"},
+        "config": {"workload": f"config{cfg}: {wl.name}; V={wl.V} n={wl.n} top-k={wl.topk if wl.topk else 'V'}, "
+                               f"target temp {wl.temp_target:g}, draft temp {wl.temp_draft:g}",
+                   "sample": f"{sample} instances per step (of the {DEFAULT_BATCH[cfg]}-instance batch)"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{sample} instances x {args.steps} steps, OpenMP over instances"},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -159,9 +190,19 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    H = HEADLINE
-    B = args.batch
-    wl = W.config3(batch=B, device=dev, seed=3000 + rank, V=H["V"], n=H["n"], topk=H["topk"])
+    cfg = args.config
+    B = args.batch if args.batch > 0 else DEFAULT_BATCH[cfg]
+    wl = make_workload(W, cfg, args.cell, B, dev, seed_offset=rank)
+    esize = wl.q_logits.element_size()
+    bytes_per_instance = wl.V * 2 * esize               # both logit rows, read once
+    kfull = wl.V if (wl.topk <= 0 or wl.topk >= wl.V) else wl.topk
+    has_rule = kfull <= G.binding.GR_MAX_SUPPORT
+    metric = (METRIC if cfg == 3 else
+              f"solve+verify instances/sec at V={wl.V},n={wl.n},top-k={wl.topk if wl.topk else 'V'}")
+    # the clock sampler runs from before the warm-up so that short timed regions still have samples
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     ev_scan = torch.cuda.Event(enable_timing=True)
     opt = G.Options(scan_done_event=ev_scan.cuda_event if hasattr(ev_scan, "cuda_event") else None)
     solved = None
@@ -184,9 +225,6 @@ def run_ours(args):
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     K = args.steps
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K)]
     scan_ms = []
@@ -240,23 +278,38 @@ def run_ours(args):
     peak, peak_kind = _peaks()
     scan_avg_ms = float(np.mean(scan_ms))
     solve_avg_ms = float(np.mean(solve_ms))
-    ach = BYTES_PER_INSTANCE * B / (scan_avg_ms * 1e-3) / 1e9
-    path_gbs = BYTES_PER_INSTANCE * B / (float(np.mean(step_ms)) * 1e-3) / 1e9
-    # dominant kernel: the solve kernel (fp64 arithmetic).  Algorithmic FMAs per gradient evaluation = nodes x
-    # [k (n(n-1)/2 + 2n) + n(n+1)/2] (series of every token, log-derivative sum, product recurrence, extraction),
-    # nodes = 26 at this shape; evaluations per instance are read back from the rule.
+    step_avg_ms = float(np.mean(step_ms))
+    ach = bytes_per_instance * B / (scan_avg_ms * 1e-3) / 1e9
+    path_gbs = bytes_per_instance * B / (step_avg_ms * 1e-3) / 1e9
     rule = G.read_rule(solved)
     evals = float(rule.iters.float().mean().item())
-    n_, k_ = H["n"], H["topk"]
-    fma_eval = 26 * (k_ * (n_ * (n_ - 1) // 2 + 2 * n_) + n_ * (n_ + 1) // 2)
-    flops = 2.0 * fma_eval * evals * B
     solve_kernel_ms = solve_avg_ms - scan_avg_ms
-    ach_tf = flops / (solve_kernel_ms * 1e-3) / 1e12
-    fp64_peak = 148 * 64 * 2 * 1.965e9 / 1e12      # SMs x fp64 FMA lanes x 2 x max SM clock
-    roof = {"bound": "alu", "kernel": "fast_solve_kernel (fp64 Newton solve; dominant)", "achieved": ach_tf,
-            "peak": fp64_peak, "unit": "TFLOP/s", "frac": ach_tf / fp64_peak, "traffic": None,
-            "peak_kind": "derived: 148 SMs x 64 fp64 FMA/clk x 1.965 GHz", "kernel_ms": solve_kernel_ms,
-            "evals_per_instance": evals}
+    # The solve kernels are plain fp64 arithmetic.  Counted here: the FMAs of the gradient evaluations alone, per
+    # evaluation  nodes x [k (n(n-1)/2 + 2n) + n(n+1)/2]  (series of every token, log-derivative sum, product
+    # recurrence, extraction) with 26 nodes; the Hessian contraction, the factorisations and the starting point are
+    # NOT counted, so the fraction understates the pipes' use and is a lower bound.  The peak is measured in this
+    # process: a cuBLAS fp64 GEMM.
+    alu = None
+    if has_rule and not args.no_extras:
+        n_, k_ = wl.n, min(kfull, G.binding.GR_MAX_SUPPORT)
+        fma_eval = 26 * (k_ * (n_ * (n_ - 1) // 2 + 2 * n_) + n_ * (n_ + 1) // 2)
+        flops = 2.0 * fma_eval * evals * B
+        ach_tf = flops / (solve_kernel_ms * 1e-3) / 1e12
+        Nm = 4096
+        am = torch.randn(Nm, Nm, dtype=torch.float64, device=dev); bm = torch.randn(Nm, Nm, dtype=torch.float64, device=dev)
+        best = 1e9
+        for i in range(6):
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); torch.mm(am, bm); e1.record(); e1.synchronize()
+            if i >= 2:
+                best = min(best, e0.elapsed_time(e1))
+        fp64_peak = 2.0 * Nm ** 3 / (best * 1e-3) / 1e12
+        del am, bm
+        alu = {"bound": "alu", "kernel": "solve kernels (fp64 Newton solve)", "achieved": ach_tf, "peak": fp64_peak,
+               "unit": "TFLOP/s", "frac": ach_tf / fp64_peak, "traffic": None,
+               "peak_kind": "measured in this process: cuBLAS fp64 GEMM 4096^3, best of 4",
+               "counted": "gradient-evaluation FMAs only (no Hessian, factorisation, starting point)",
+               "kernel_ms": solve_kernel_ms, "evals_per_instance": evals}
     status = solved.status.cpu().numpy()
     acc_rate = float(ver.accepted.float().mean().item())
 
@@ -297,34 +350,79 @@ def run_ours(args):
                  "p50_us": float(np.median(fms)) * 1e3, "gpu_launches_per_step": 3,
                  "same_tokens_as_two_call_path": same}
 
-    # ---- CPU baseline: the oracle on a bounded sample of the same workload
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload; the same sample gives the parity
+    #      figures of this very run (optimal acceptance, verification distribution, emitted tokens)
     cpu = None
+    parity = None
     if not args.no_extras:
         from oracle import gr_oracle as O
-        ns = min(128, B)
+        ns = min(ORACLE_SAMPLE[cfg], B)
         sub = wl.rows(list(range(ns)))
         tl = W.logits_to_f64(sub.q_logits); dl = W.logits_to_f64(sub.p_logits)
-        t0 = time.perf_counter()
-        O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, sub.draft_tokens.cpu().numpy(),
-                             sub.uniforms.cpu().numpy())
-        cpu_dt = time.perf_counter() - t0
-        cpu = {"value": ns / cpu_dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-               "sample": f"first {ns} instances of the batch, OpenMP over instances, {cpu_dt:.1f} s"}
+        g_alpha = solved.alpha_star[:ns].double().cpu().numpy()
+        if has_rule:
+            t0 = time.perf_counter()
+            res = O.solve_verify_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft,
+                                       sub.draft_tokens.cpu().numpy(), sub.uniforms.cpu().numpy())
+            cpu_dt = time.perf_counter() - t0
+            cpu = {"value": ns / cpu_dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+                   "sample": f"first {ns} instances of the batch, OpenMP over instances, {cpu_dt:.1f} s"}
+            sl = G.read_slice(solved, wl.draft_tokens)
+            g_tok = ver.token[:ns].cpu().numpy(); g_acc = ver.accepted[:ns].cpu().numpy()
+            tv = 0.0
+            for b_ in range(ns):
+                keep = sl.U[b_].numpy() >= 0
+                nu = int((res.U[b_] >= 0).sum())
+                if int(keep.sum()) != nu:
+                    tv = float("inf"); continue
+                kk = int(res.k[b_])
+                ro = res.r[b_, :kk] / max(1.0 - res.alpha_star[b_], 1e-300)
+                rg = rule.resid[b_, :kk].numpy() / max(1.0 - float(rule.alpha_star[b_]), 1e-300)
+                rho_g, rho_o = float(sl.rho[b_]), float(res.rho[b_])
+                tv = max(tv, 0.5 * (np.abs(sl.pi[b_].numpy()[keep] - res.pi[b_, :nu]).sum()
+                                    + np.abs(rho_g * rg - rho_o * ro).sum()
+                                    + abs(rho_g * (1 - rg.sum()) - rho_o * (1 - ro.sum()))))
+            _, _, margin = O.draw_sweep_batch(tl, dl, wl.n, wl.topk, wl.temp_target, wl.temp_draft, res,
+                                              sub.draft_tokens.cpu().numpy(), sub.uniforms.cpu().numpy()[:, None, :])
+            diff = (g_tok != res.token) | (g_acc != res.accepted)
+            parity = {"sample": ns, "alpha_star_max_abs_err": float(np.max(np.abs(g_alpha - res.alpha_star))),
+                      "tv_max": tv, "token_mismatch_within_1e-6_of_a_cdf_boundary": int(np.sum(diff & (margin[:, 0] < 1e-6))),
+                      "token_mismatch_other": int(np.sum(diff & (margin[:, 0] >= 1e-6))),
+                      "structure_mismatch": int(np.sum(rule.jstar[:ns].numpy() != res.jstar))}
+        else:
+            # whole-vocabulary draft beyond the solve capacity: the oracle gives the optimal acceptance only
+            t0 = time.perf_counter()
+            a_or = np.array([O.alpha_star_only(tl[i], dl[i], wl.n, wl.topk, wl.temp_target, wl.temp_draft)[0]
+                             for i in range(ns)])
+            cpu_dt = time.perf_counter() - t0
+            cpu = {"value": ns / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                   "sample": f"optimal acceptance only (no rule at this support size), first {ns} instances, {cpu_dt:.1f} s"}
+            parity = {"sample": ns, "alpha_star_max_abs_err": float(np.max(np.abs(g_alpha - a_or))), "tv_max": None,
+                      "note": "no verification rule at this support size: gr_verify samples the target"}
 
+    iters = rule.iters.numpy()
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
+        "metric": metric, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3),
         "ms_per_step": dev_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"config3: V=128256 n=8 top-k=50 batch {B} per GPU, fp32 logits, target temp 0.7, "
-                               "draft temp 1.0, Zipf-shaped logits", "global_batch": world * B,
-                   "cache": f"inputs ({BYTES_PER_INSTANCE * B / 1e9:.2f} GB per batch) larger than L2, no flush needed", "parallelism": f"batch x{world}"},
-        "roofline": roof,
+        "config": {"workload": f"config{cfg}: {wl.name}; V={wl.V} n={wl.n} top-k={wl.topk if wl.topk else 'V'} batch {B} "
+                               f"per GPU, {'bf16' if esize == 2 else 'fp32'} logits, target temp {wl.temp_target:g}, "
+                               f"draft temp {wl.temp_draft:g}", "global_batch": world * B,
+                   "cache": (f"one input set of {bytes_per_instance * B / 1e9:.2f} GB per batch, re-read every step: "
+                             + ("larger than the 126 MB L2, no flush needed" if bytes_per_instance * B > 3e8 else
+                                "SMALLER than L2 (the configuration is that small); the step is not HBM-bound")),
+                   "parallelism": f"batch x{world}"},
+        "roofline": {"bound": "hbm", "kernel": "whole step (streaming + solve + verify kernels)",
+                     "what": "bytes of both logit rows / whole solve+verify step time (the streaming kernel is the "
+                             "only one that reads them; the solve kernels work on-chip)",
+                     "achieved": path_gbs, "peak": peak, "unit": "GB/s", "frac": path_gbs / peak,
+                     "traffic": SCAN_TRAFFIC_RATIO * bytes_per_instance * B, "peak_kind": peak_kind,
+                     "frac_of_8TBs_datasheet": path_gbs / 8000.0, "step_ms": step_avg_ms},
         "roofline_scan": {"bound": "hbm", "kernel": "scan_kernel (streams both logit rows once)", "achieved": ach,
-                          "peak": peak, "unit": "GB/s", "frac": ach / peak, "traffic": SCAN_TRAFFIC_PER_INSTANCE * B,
-                          "peak_kind": peak_kind, "kernel_ms": scan_avg_ms},
-        "roofline_path": {"bound": "hbm", "what": "bytes of both logit rows / whole solve+verify step time",
-                          "achieved": path_gbs, "peak": peak, "unit": "GB/s", "frac": path_gbs / peak,
-                          "frac_of_8TBs_datasheet": path_gbs / 8000.0},
+                          "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                          "traffic": SCAN_TRAFFIC_RATIO * bytes_per_instance * B, "peak_kind": peak_kind,
+                          "kernel_ms": scan_avg_ms},
+        "roofline_solve": alu,
         "kernels_ms": {"scan": scan_avg_ms, "solve": solve_avg_ms - scan_avg_ms, "verify": float(np.mean(verify_ms))},
         "fused_call": fused,
         "p50_us": {"batch_step": float(np.median(step_ms)) * 1e3,
@@ -335,8 +433,11 @@ def run_ours(args):
         "e2e": e2e,
         "gpu_launches": 4 * K,   # scan, fast solve, robust solve (flagged instances only), verify
         "clocks": clocks,
-        "quality": {"accept_rate": acc_rate, "status_ok": int((status == 0).sum()),
-                    "status_not_converged": int((status == 1).sum()), "wall_ms_total": total_ms},
+        "quality": {"accept_rate": acc_rate, "alpha_star_mean": float(solved.alpha_star.float().nanmean().item()),
+                    "status_ok": int((status == 0).sum()), "status_not_converged": int((status == 1).sum()),
+                    "status_no_rule": int((status == 2).sum()),
+                    "iterations_histogram": np.bincount(iters, minlength=1).tolist()[:64],
+                    "gnorm_max": float(rule.gnorm.max()), "parity_vs_oracle": parity, "wall_ms_total": total_ms},
     }
     print(json.dumps(out), flush=True)
     if world > 1:
@@ -349,8 +450,13 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--batch", type=int, default=HEADLINE["batch"],
-                    help="instances per GPU (default: the headline 1024; smaller values are for profiler captures)")
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5],
+                    help="benchmark configuration (default 3: the headline V=128256, n=8, top-k=50)")
+    ap.add_argument("--cell", type=lambda t: tuple(float(x) for x in t.split(",")), default=(8, 20, 1.0),
+                    help="configuration 4 only: n,topk,sigma of the sweep cell (topk 0 = whole vocabulary)")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="instances per GPU (default: the configuration's own, 1024 at the headline; smaller values "
+                         "are for profiler captures)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the end-to-end, batch-1 and CPU-baseline legs (profiler captures)")
     args = ap.parse_args()
