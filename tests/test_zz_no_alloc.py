@@ -57,9 +57,36 @@ def test_static_scratch_matches_caller_workspace_on_two_calls_in_a_row():
     _same(W.config3(batch=20, device="cuda", V=40000, n=4, topk=24))
 
 
-def test_static_scratch_rejects_batches_beyond_its_capacity():
+def test_static_call_leaves_free_device_memory_unchanged():
+    """What the entry point is for: after its first call on the device (which looks up the built-in array's
+    address) a call allocates nothing.  Free device memory as the driver reports it is the same before and after
+    a call whose outputs were allocated beforehand."""
+    build_library()
+    wl = W.config2(batch=32, device="cuda", V=9000)
+    _static_solve(wl)                      # first call on this device: set-up
+    B = wl.batch
+    dev = wl.q_logits.device
+    params = torch.empty(G.gr_params_bytes(wl.V, wl.n, wl.topk, B), dtype=torch.uint8, device=dev)
+    alpha = torch.empty(B, dtype=torch.float32, device=dev)
+    status = torch.empty(B, dtype=torch.int32, device=dev)
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        rc = G.gr_solve_static(wl.q_logits.data_ptr(), wl.p_logits.data_ptr(), G.GR_F32, wl.V, wl.n, wl.topk,
+                               wl.temp_target, wl.temp_draft, B, None, params.data_ptr(), alpha.data_ptr(),
+                               status.data_ptr(), int(torch.cuda.current_stream().cuda_stream))
+        assert rc == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    assert status.cpu().tolist() == [G.GR_OK] * B
+
+
+def test_static_scratch_rejects_what_it_cannot_hold():
     build_library()
     A = 1 << 20
     rc = G.gr_solve_static(A, A, G.GR_F32, 1000, 2, 8, 1.0, 1.0, G.GR_STATIC_MAX_BATCH + 1, None, A, A, A, 0)
     assert rc == -5 and "capacity" in G.gr_strerror(rc)
     assert G.gr_solve_static(A, A, G.GR_F32, 1000, 2, 8, 1.0, 1.0, 0, None, A, A, A, 0) == 0
+    # an untruncated draft on a vocabulary beyond the solve capacity needs a per-row sort buffer the scratch lacks
+    assert G.gr_solve_static(A, A, G.GR_F32, 100000, 2, 0, 1.0, 1.0, 2, None, A, A, A, 0) == -5
