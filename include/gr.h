@@ -46,6 +46,8 @@ extern "C" {
 #define GR_STALE_PARAMS          5  /* params block was not written by gr_solve for this shape            */
 #define GR_PARTIAL_RULE          6  /* params written by gr_solve_verify: only the system its drafted tuple
                                        selects was solved; gr_verify refuses such a block (token -1)       */
+#define GR_CHECK_FAILED          7  /* bounds-checked build of the library only: a kernel skipped an access
+                                       outside an array's extent while it worked on this instance          */
 
 /* host-side argument errors (return values) */
 #define GR_E_INVALID   (-1)  /* a size, temperature or option is out of range */

@@ -9,6 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libgr_b200.so")
+LIB_CHECK = os.path.join(HERE, "libgr_b200_check.so")      # the bounds-checked build (-DGR_CHECK)
 OBJ = os.path.join(HERE, "_build")
 SOURCES = ["gr_api.cu", "gr_alpha.cu", "gr_static.cu", "gr_scan.cu", "gr_solve.cu", "gr_fast.cu", "gr_fast_n4.cu", "gr_fast_n8.cu",
            "gr_fast_n16.cu", "gr_fast_w8.cu", "gr_fast_w16.cu", "gr_fullsort.cu", "gr_verify.cu"]
@@ -23,22 +24,29 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def needs_build() -> bool:
-    if not os.path.exists(LIB):
+def needs_build(check: bool = False) -> bool:
+    lib = LIB_CHECK if check else LIB
+    if not os.path.exists(lib):
         return True
-    t = os.path.getmtime(LIB)
+    t = os.path.getmtime(lib)
     deps = [os.path.join(CSRC, s) for s in SOURCES] + HEADERS
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
+def build_library(force: bool = False, verbose: bool = False, check: bool = False) -> str:
     """Compile each source to an object (in parallel; objects newer than every source and header are kept),
-    then link the shared library."""
-    if not force and not needs_build():
+    then link the shared library.  check=True builds the bounds-checked variant (-DGR_CHECK: every access through a
+    pointer into shared memory, the workspace records or the params block is range-checked, an out-of-range access
+    is skipped and reported as status GR_CHECK_FAILED) into a library file of its own; it is for tests only."""
+    LIB = LIB_CHECK if check else globals()["LIB"]
+    OBJ = globals()["OBJ"] + ("_check" if check else "")
+    if not force and not needs_build(check):
         return LIB
     os.makedirs(OBJ, exist_ok=True)
     flags = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-Xcompiler", "-fPIC",
              "-I", os.path.join(ROOT, "include"), "-I", CSRC]
+    if check:
+        flags += ["-DGR_CHECK"]
     if verbose:
         flags += ["-Xptxas", "-v"]
     hdr_time = max(os.path.getmtime(h) for h in HEADERS)

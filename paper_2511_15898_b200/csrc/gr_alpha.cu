@@ -34,12 +34,12 @@ alpha_kernel(const char* __restrict__ ws, int V, int topk, double temp_t, double
         a_i = (double)wv.tl[tid] / temp_t;
         b_i = (double)wv.dl[tid] / temp_d;
     }
-    const double bmax = block_reduce_max(tid < k ? b_i : -1.0e300, s_red);
-    const double bsum = block_reduce_sum(tid < k ? exp(b_i - bmax) : 0.0, s_red);
+    const double bmax = block_reduce_max(tid < k ? b_i : -1.0e300, GR_MKPTR(double, s_red, 32, nullptr));
+    const double bsum = block_reduce_sum(tid < k ? exp(b_i - bmax) : 0.0, GR_MKPTR(double, s_red, 32, nullptr));
     const double lse_d = bmax + log(bsum);
     if (kfull == V) {
-        const double amax = block_reduce_max(tid < k ? a_i : -1.0e300, s_red);
-        const double asum = block_reduce_sum(tid < k ? exp(a_i - amax) : 0.0, s_red);
+        const double amax = block_reduce_max(tid < k ? a_i : -1.0e300, GR_MKPTR(double, s_red, 32, nullptr));
+        const double asum = block_reduce_sum(tid < k ? exp(a_i - amax) : 0.0, GR_MKPTR(double, s_red, 32, nullptr));
         lse_t = amax + log(asum);
     }
     // ratio order: decreasing log-ratio, equal keys by smaller id (Sec. 5.1)

@@ -187,6 +187,37 @@ int gr_read_slice(const void* params, const int* draft_tokens, int batch, int n,
     return GR_OK;
 }
 
+#ifdef GR_CHECK
+// Bounds-checked build only: exercises the checked pointer itself.  A kernel reads and writes a 4-entry shared
+// array through it at indices -1 .. 4; out[0] = number of accesses that were skipped and flagged (expected 2),
+// out[1] = sum of what the in-range reads returned (expected 0+1+2+3), out[2] = the values the skipped reads gave.
+namespace gr {
+__global__ void check_selftest_kernel(int* out)
+{
+    __shared__ int arr[4];
+    __shared__ int flag;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 4; i++) arr[i] = i;
+        int skipped = 0, sum = 0, ghost = 0;
+        for (int i = -1; i <= 4; i++) {
+            flag = 0;
+            CkPtr<int> p(arr, 4, &flag);
+            const int v = p[i];
+            p[i] = v;                       // a skipped write must not land anywhere
+            if (flag) { skipped++; ghost += v; } else sum += v;
+        }
+        out[0] = skipped; out[1] = sum; out[2] = ghost;
+        out[3] = arr[0] + arr[1] + arr[2] + arr[3];
+    }
+}
+}  // namespace gr
+int gr_check_selftest(int* out_device, void* stream)
+{
+    gr::check_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(out_device);
+    return cudaPeekAtLastError() == cudaSuccess ? GR_OK : GR_E_LAUNCH;
+}
+#endif
+
 const char* gr_strerror(int code)
 {
     switch (code) {
@@ -197,6 +228,7 @@ const char* gr_strerror(int code)
         case GR_DRAFT_OUT_OF_SUPPORT: return "drafted token outside the draft support";
         case GR_STALE_PARAMS: return "params block was not written by gr_solve";
         case GR_PARTIAL_RULE: return "rule solved only for the drafts given to gr_solve_verify";
+        case GR_CHECK_FAILED: return "bounds-checked build: an out-of-range access was skipped";
         case GR_E_INVALID: return "invalid size, temperature or option";
         case GR_E_NULL: return "required pointer is NULL";
         case GR_E_ALIGN: return "pointer is not 16-byte aligned";

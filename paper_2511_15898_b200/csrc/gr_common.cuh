@@ -8,6 +8,52 @@
 
 namespace gr {
 
+// ---- Bounds-checked build.  Compiled with -DGR_CHECK (paper_2511_15898_b200.build.build_library(check=True), a
+// separate library file) every pointer into shared memory, into the workspace records and into the params block
+// carries its extent: an access outside it is SKIPPED (a read gives 0) and raises a per-CTA flag, which the kernel
+// turns into the instance's status GR_CHECK_FAILED.  It stands in for a memory checker on machines where none may
+// run; nothing traps or asserts.  Without the macro the same names are plain pointers and cost nothing.
+#ifdef GR_CHECK
+template <class T> struct CkNonConst { typedef T type; };
+template <class T> struct CkNonConst<const T> { typedef T type; };
+template <class T>
+struct CkPtr {
+    T* p; long long n; int* bad;
+    mutable typename CkNonConst<T>::type sink;
+    __host__ __device__ CkPtr() : p(nullptr), n(0), bad(nullptr), sink() {}
+    __host__ __device__ CkPtr(T* p_, long long n_, int* bad_) : p(p_), n(n_), bad(bad_), sink() {}
+    template <class U> __host__ __device__ CkPtr(const CkPtr<U>& o) : p(o.p), n(o.n), bad(o.bad), sink() {}
+    __device__ T& operator[](long long i) const {
+        if (i >= 0 && i < n) return p[i];
+        if (bad) *bad = 1;
+        sink = typename CkNonConst<T>::type();
+        return sink;
+    }
+    __device__ T& operator*() const { return (*this)[0]; }
+    __host__ __device__ CkPtr operator+(long long k) const { return CkPtr(p + k, n - k, bad); }
+    __host__ __device__ CkPtr operator-(long long k) const { return CkPtr(p - k, n + k, bad); }
+    template <class U> __host__ __device__ CkPtr<U> as() const {
+        return CkPtr<U>(reinterpret_cast<U*>(p), n * (long long)sizeof(T) / (long long)sizeof(U), bad);
+    }
+};
+#define GR_PTR(T) ::gr::CkPtr<T>
+#define GR_MKPTR(T, ptr, count, flag) ::gr::CkPtr<T>((ptr), (count), (flag))
+#define GR_PCAST(T, ptr) ((ptr).template as<T>())
+#define GR_CHECK_FLAG_DECL __shared__ int s_check_flag
+#define GR_CHECK_FLAG (&s_check_flag)
+#define GR_CHECK_FLAG_INIT do { if (threadIdx.x == 0) s_check_flag = 0; __syncthreads(); } while (0)
+#define GR_CHECK_VALUE (s_check_flag)
+#else
+template <class T> using RawPtr = T*;       // (an alias, so that "GR_PTR(double) a, b;" declares two pointers)
+#define GR_PTR(T) ::gr::RawPtr<T>
+#define GR_MKPTR(T, ptr, count, flag) (ptr)
+#define GR_PCAST(T, ptr) (reinterpret_cast<T*>(ptr))
+#define GR_CHECK_FLAG_DECL
+#define GR_CHECK_FLAG (nullptr)
+#define GR_CHECK_FLAG_INIT do { } while (0)
+#define GR_CHECK_VALUE (0)
+#endif
+
 constexpr int kMaxSupport = GR_MAX_SUPPORT;   // largest support the convex programs are solved on
 constexpr int kMaxDrafts = GR_MAX_DRAFTS;     // largest n
 constexpr int kChunk = 1024;                  // elements per chunk of the target-row mass table
@@ -49,18 +95,20 @@ __host__ __device__ inline int params_stride(int V, int topk) {
     return round16((int)sizeof(Header) + kcap_of(V, topk) * 32 + nchcap_of(V) * 8);
 }
 struct ParamView {
-    Header* h; int* id; int* blk; double* w; double* r; double* p; float2* chunk;
+    Header* h; GR_PTR(int) id; GR_PTR(int) blk; GR_PTR(double) w; GR_PTR(double) r; GR_PTR(double) p; GR_PTR(float2) chunk;
 };
-__host__ __device__ inline ParamView view_params(void* base, int kcap) {
+// (V and `flag` only matter to the bounds-checked build: extent of the chunk table, where to report)
+__host__ __device__ inline ParamView view_params(void* base, int kcap, int V = 1 << 21, int* flag = nullptr) {
     ParamView v;
     char* c = (char*)base;
     v.h = (Header*)c; c += sizeof(Header);
-    v.w = (double*)c; c += (size_t)kcap * 8;
-    v.r = (double*)c; c += (size_t)kcap * 8;
-    v.p = (double*)c; c += (size_t)kcap * 8;
-    v.id = (int*)c; c += (size_t)kcap * 4;
-    v.blk = (int*)c; c += (size_t)kcap * 4;
-    v.chunk = (float2*)c;
+    v.w = GR_MKPTR(double, (double*)c, kcap, flag); c += (size_t)kcap * 8;
+    v.r = GR_MKPTR(double, (double*)c, kcap, flag); c += (size_t)kcap * 8;
+    v.p = GR_MKPTR(double, (double*)c, kcap, flag); c += (size_t)kcap * 8;
+    v.id = GR_MKPTR(int, (int*)c, kcap, flag); c += (size_t)kcap * 4;
+    v.blk = GR_MKPTR(int, (int*)c, kcap, flag); c += (size_t)kcap * 4;
+    v.chunk = GR_MKPTR(float2, (float2*)c, nchcap_of(V), flag);
+    (void)V; (void)flag;
     return v;
 }
 
@@ -70,7 +118,8 @@ struct __align__(16) WsHeader {
     double lse_d;        // same for the whole draft row (only when the support is the whole vocabulary)
     int count;           // entries that follow (the support, k of them)
     int bad;             // 1 when a non-finite logit was met
-    int pad[2];
+    int check;           // bounds-checked build: the streaming kernel skipped an out-of-range access on this row
+    int pad;
 };
 // then: int id[kMaxSupport]; float dl[kMaxSupport]; float tl[kMaxSupport];
 __host__ __device__ inline int ws_stride() { return (int)sizeof(WsHeader) + kMaxSupport * 12; }

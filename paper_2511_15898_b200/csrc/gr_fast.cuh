@@ -53,7 +53,7 @@ constexpr int kFSweeps = 5;           // fixed-point sweeps of the starting poin
 struct FastLayout {
     int KP;
     int d, tg, p, r, key, psi, Dr, alpha, alpha_prev, delta, w, g, g2, col, gw, g2w, tq, cq, scal, uni;
-    int jacc_bytes_off, ints, total_bytes;
+    int jacc_bytes_off, ints, total_bytes, uni_doubles;
     __host__ __device__ FastLayout(int KP_, int NT) : KP(KP_) {
         int o = 0;
         d = o; o += KP; tg = o; o += KP; p = o; o += KP; r = o; o += KP; key = o; o += KP;
@@ -67,7 +67,8 @@ struct FastLayout {
         // union: staging of the Hessian operands (two float arrays [kJC * NT][kMS]) / vectors of the Newton step
         const int stage_doubles = (2 * kJC * NT * kMS * 4 + 7) / 8;
         const int jmat_doubles = 2 * (kMP + 4) + 2 * kMP;    // (floats, so twice what is needed) pivot row / column buffers
-        o += stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
+        uni_doubles = stage_doubles > jmat_doubles ? stage_doubles : jmat_doubles;
+        o += uni_doubles;
         jacc_bytes_off = o * 8;                       // float [kMP][kMP] accumulator of the contraction
         o += (kMP * (kMP + 1) + 1) / 2;
         ints = o * 8;
@@ -77,10 +78,9 @@ struct FastLayout {
 static inline int fast_smem_bytes(int KP, int NT) { return FastLayout(KP, NT).total_bytes; }
 
 struct FSm {
-    double *d, *tg, *p, *r, *key, *psi, *Dr, *alpha, *alpha_prev, *delta, *w, *g, *g2, *col, *gw, *g2w, *tq, *cq,
-        *scal, *J;
-    float *AS, *HS, *Jacc;
-    int *id, *blk, *itmp, *trunc;
+    GR_PTR(double) d, tg, p, r, key, psi, Dr, alpha, alpha_prev, delta, w, g, g2, col, gw, g2w, tq, cq, scal, J;
+    GR_PTR(float) AS, HS, Jacc;
+    GR_PTR(int) id, blk, itmp, trunc;
     int KP;
 };
 enum { SC_Q = 0, SC_FAIL = 1, SC_RED = 8 };
@@ -219,8 +219,8 @@ __device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
         if (i0 >= m || l0 >= m) continue;
         float c0 = 0.f, c1 = 0.f, c2 = 0.f, c3 = 0.f;
         for (int k0 = 0; k0 < K8; k0 += 8) {
-            const float* Ap = sm.AS + (k0 + tig) * kMS + i0 + gid;
-            const float* Bp = sm.HS + (k0 + tig) * kMS + l0 + gid;
+            GR_PTR(const float) Ap = sm.AS + ((k0 + tig) * kMS + i0 + gid);
+            GR_PTR(const float) Bp = sm.HS + ((k0 + tig) * kMS + l0 + gid);
             const float fa[4] = {Ap[0], Ap[8], Ap[4 * kMS], Ap[4 * kMS + 8]};
             const float fb[2] = {Bp[0], Bp[4 * kMS]};
             if (kSplit) {
@@ -243,7 +243,7 @@ __device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
                          __float_as_uint(fa[3]), __float_as_uint(fb[0]), __float_as_uint(fb[1]));
             }
         }
-        float* J0 = sm.Jacc + (i0 + gid) * kJS + l0 + 2 * tig;
+        GR_PTR(float) J0 = sm.Jacc + ((i0 + gid) * kJS + l0 + 2 * tig);
         J0[0] += c0; J0[1] += c1;
         J0[8 * kJS] += c2; J0[8 * kJS + 1] += c3;
     }
@@ -253,7 +253,7 @@ __device__ __forceinline__ void hess_chunk(const FSm& sm, int K8, int m)
 // The contraction takes every jstride-th node (weights scaled by jstride).
 // Node abscissae / weights are in sm.tq / sm.cq, their number in sm.scal[SC_Q].
 template <int NT, int TPL>
-__device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double hmass, bool want_jac, int jstride)
+__device__ void fast_eval(const FSm& sm, int m, int n, GR_PTR(const double) d, double hmass, bool want_jac, int jstride)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, KP = sm.KP;
     const int Q = (int)sm.scal[SC_Q];
@@ -348,8 +348,8 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
                     // are zero (they pad the contraction length to a multiple of the MMA depth).
                     const int j = lane + 32 * tt;
                     const double sa = (double)jstride * cq * t * u;
-                    float* as = sm.AS + slot * NT * kMS + j;
-                    float* hs = sm.HS + slot * NT * kMS + j;
+                    GR_PTR(float) as = sm.AS + (slot * NT * kMS + j);
+                    GR_PTR(float) hs = sm.HS + (slot * NT * kMS + j);
                     if (n == NT) {
                         // full series length: fixed rows, each A consumed as soon as it is formed
 #pragma unroll
@@ -414,7 +414,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, const double* d, double h
 static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
 {
     const int tid = threadIdx.x;
-    double* red = sm.scal + SC_RED;
+    GR_PTR(double) red = sm.scal + SC_RED;
     double a = 0.0;
     if (tid < m) { a = sm.alpha[tid]; sm.w[tid] = exp(a); }
     // extreme alphas in one pass (they give the extreme weights)
@@ -454,13 +454,13 @@ static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double 
 // steers the iteration (the fp64 gradient decides convergence) and the Hessian was accumulated in fp32.
 // Matrix: off-diagonal -Jacc (lower triangle), diagonal g - g2, plus `add` everywhere.  Writes the step
 // into sm.delta; sets SC_FAIL when a pivot is not positive.
-static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs, double add)
+static __device__ void fast_newton_step(const FSm& sm, int m, GR_PTR(const double) rhs, double add)
 {
     const int tid = threadIdx.x;
-    float* Jm = sm.Jacc;
-    float* yv = reinterpret_cast<float*>(sm.J);        // [kMP] working right-hand side
-    float* yf = yv + kMP;                              // [kMP] forward-substituted right-hand side, then the solution
-    float* dg = yf + kMP;                              // [kMP] diagonal of the factor
+    GR_PTR(float) Jm = sm.Jacc;
+    GR_PTR(float) yv = GR_PCAST(float, sm.J);          // [kMP] working right-hand side
+    GR_PTR(float) yf = yv + kMP;                       // [kMP] forward-substituted right-hand side, then the solution
+    GR_PTR(float) dg = yf + kMP;                       // [kMP] diagonal of the factor
     const float addf = (float)add;
     for (int e = tid; e < m * kMP; e += kFT) {
         const int i = e / kMP, l = e & (kMP - 1);
@@ -556,8 +556,8 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
                     const float fa[4] = {oa ? -Jm[ra * kJS + j0 + tig] : 0.f, ob ? -Jm[rb * kJS + j0 + tig] : 0.f,
                                          oa ? -Jm[ra * kJS + j0 + tig + 4] : 0.f, ob ? -Jm[rb * kJS + j0 + tig + 4] : 0.f};
                     const float fb[2] = {oc ? Jm[cb * kJS + j0 + tig] : 0.f, oc ? Jm[cb * kJS + j0 + tig + 4] : 0.f};
-                    float* C0 = Jm + ra * kJS + l0 + 2 * tig;
-                    float* C1 = Jm + rb * kJS + l0 + 2 * tig;
+                    GR_PTR(float) C0 = Jm + (ra * kJS + l0 + 2 * tig);
+                    GR_PTR(float) C1 = Jm + (rb * kJS + l0 + 2 * tig);
                     float c0 = oa ? C0[0] : 0.f, c1 = oa ? C0[1] : 0.f, c2 = ob ? C1[0] : 0.f, c3 = ob ? C1[1] : 0.f;
                     uint32_t ah[4], al[4], bh[2], bl[2];
 #pragma unroll
@@ -649,11 +649,11 @@ static __device__ void fast_newton_step(const FSm& sm, int m, const double* rhs,
 
 // Newton iteration for one system.  On return sm.w holds exp(alpha) at the last evaluated point.
 template <int NT, int TPL>
-__device__ int fast_system(const FSm& sm, int m, int n, const double* d, const double* rhs, double hmass, int slack,
-                           double tol, int max_iters, double qstep, double* gnorm, int* iters)
+__device__ int fast_system(const FSm& sm, int m, int n, GR_PTR(const double) d, GR_PTR(const double) rhs, double hmass,
+                           int slack, double tol, int max_iters, double qstep, double* gnorm, int* iters)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    double* red = sm.scal + SC_RED;
+    GR_PTR(double) red = sm.scal + SC_RED;
     // ---- mean-field starting point: token i wins the share w_i / (slack + w_i + S_i) of the tuples that
     //      contain it, S_i = expected weight of the other drafted tokens given that i was drafted
     const double T = hmass + block_reduce_sum(tid < m ? d[tid] : 0.0, red);
@@ -688,20 +688,20 @@ __device__ int fast_system(const FSm& sm, int m, int n, const double* d, const d
     // fp32: it is a starting point.
     if (tid < m) { sm.g2[tid] = 1.0 / ci; sm.g[tid] = (slack ? 1.0 : 0.0) + wi; }
     __syncthreads();
-    float* part = sm.AS;                              // [kFW][kMP] partial sums (the staging area is idle here)
+    GR_PTR(float) part = sm.AS;                       // [kFW][kMP] partial sums (the staging area is idle here)
     for (int sweep = 0; sweep < kFSweeps; sweep++) {
         // lane = rows lane, lane + 32, ...; warp = a contiguous share of the columns: no shuffles, independent sums
         {
             const int chunk = (m + kFW - 1) / kFW;
             const int jlo = warp * chunk, jhi = min(m, jlo + chunk);
             float Ar[kRL], cr[kRL], sa[kRL], sb[kRL];
-            const float* row[kRL];
+            GR_PTR(const float) row[kRL];
 #pragma unroll
             for (int u = 0; u < kRL; u++) {
                 const int r = lane + 32 * u;
                 const bool on = r < m;
                 Ar[u] = on ? (float)sm.g[r] : 1.f; cr[u] = on ? (float)sm.g2[r] : 0.f;
-                row[u] = sm.Jacc + (on ? r : 0) * kJS;
+                row[u] = sm.Jacc + ((on ? r : 0) * kJS);
                 sa[u] = 0.f; sb[u] = 0.f;
             }
             int j = jlo;
@@ -819,17 +819,19 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_sel;
+    GR_CHECK_FLAG_DECL;
+    GR_CHECK_FLAG_INIT;
     const bool fused = fa.draft != nullptr;
     const int tid = threadIdx.x;
     const long long b = blockIdx.x;
     char* pb = params + (size_t)b * pstride;
-    ParamView pv = view_params(pb, kcap);
-    const WsView wv = view_ws(ws, b);
+    ParamView pv = view_params(pb, kcap, V, GR_CHECK_FLAG);
+    const WsView wv = view_ws(ws, b, GR_CHECK_FLAG);
     if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
         if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
         if (fused) {
             __syncthreads();
-            fused_draw(fa, pv.h, b, n, smem_raw);
+            fused_draw(fa, pv.h, b, n, smem_raw, GR_CHECK_FLAG);
         }
         return;
     }
@@ -837,16 +839,26 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     FastLayout L(KP, NT);
     double* base = reinterpret_cast<double*>(smem_raw);
     FSm sm;
-    sm.d = base + L.d; sm.tg = base + L.tg; sm.p = base + L.p; sm.r = base + L.r; sm.key = base + L.key;
-    sm.psi = base + L.psi; sm.Dr = base + L.Dr; sm.alpha = base + L.alpha; sm.alpha_prev = base + L.alpha_prev;
-    sm.delta = base + L.delta; sm.w = base + L.w; sm.g = base + L.g; sm.g2 = base + L.g2; sm.col = base + L.col;
-    sm.gw = base + L.gw; sm.g2w = base + L.g2w; sm.tq = base + L.tq; sm.cq = base + L.cq; sm.scal = base + L.scal;
-    sm.J = base + L.uni;
-    sm.AS = reinterpret_cast<float*>(base + L.uni);
-    sm.HS = sm.AS + kJC * NT * kMS;
-    sm.Jacc = reinterpret_cast<float*>(smem_raw + L.jacc_bytes_off);
+    int* const ck = GR_CHECK_FLAG;
+    (void)ck;
+    sm.d = GR_MKPTR(double, base + L.d, KP, ck); sm.tg = GR_MKPTR(double, base + L.tg, KP, ck);
+    sm.p = GR_MKPTR(double, base + L.p, KP, ck); sm.r = GR_MKPTR(double, base + L.r, KP, ck);
+    sm.key = GR_MKPTR(double, base + L.key, KP, ck);
+    sm.psi = GR_MKPTR(double, base + L.psi, KP + 4, ck); sm.Dr = GR_MKPTR(double, base + L.Dr, KP + 4, ck);
+    sm.alpha = GR_MKPTR(double, base + L.alpha, KP, ck); sm.alpha_prev = GR_MKPTR(double, base + L.alpha_prev, KP, ck);
+    sm.delta = GR_MKPTR(double, base + L.delta, KP, ck); sm.w = GR_MKPTR(double, base + L.w, KP, ck);
+    sm.g = GR_MKPTR(double, base + L.g, KP, ck); sm.g2 = GR_MKPTR(double, base + L.g2, KP, ck);
+    sm.col = GR_MKPTR(double, base + L.col, kMP, ck);
+    sm.gw = GR_MKPTR(double, base + L.gw, kFW * KP, ck); sm.g2w = GR_MKPTR(double, base + L.g2w, kFW * KP, ck);
+    sm.tq = GR_MKPTR(double, base + L.tq, kFMaxNodes, ck); sm.cq = GR_MKPTR(double, base + L.cq, kFMaxNodes, ck);
+    sm.scal = GR_MKPTR(double, base + L.scal, 32, ck);
+    sm.J = GR_MKPTR(double, base + L.uni, L.uni_doubles, ck);
+    sm.AS = GR_MKPTR(float, reinterpret_cast<float*>(base + L.uni), kJC * NT * kMS, ck);
+    sm.HS = GR_MKPTR(float, reinterpret_cast<float*>(base + L.uni) + kJC * NT * kMS, kJC * NT * kMS, ck);
+    sm.Jacc = GR_MKPTR(float, reinterpret_cast<float*>(smem_raw + L.jacc_bytes_off), kMP * kJS, ck);
     int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
-    sm.id = ib; sm.blk = ib + KP; sm.itmp = ib + 2 * KP; sm.trunc = ib + 3 * KP;
+    sm.id = GR_MKPTR(int, ib, KP, ck); sm.blk = GR_MKPTR(int, ib + KP, KP, ck);
+    sm.itmp = GR_MKPTR(int, ib + 2 * KP, KP, ck); sm.trunc = GR_MKPTR(int, ib + 3 * KP, KP, ck);
     sm.KP = KP;
     PrepSm ps;
     ps.d = sm.d; ps.tg = sm.tg; ps.p = sm.p; ps.r = sm.r; ps.key = sm.key; ps.psi = sm.psi; ps.Dr = sm.Dr;
@@ -864,7 +876,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
         truncation_sets(ps, sm.trunc, sm.itmp, k, jstar, n, tau);
         tol = 5.0 * tau;
     }
-    double* dT = sm.key; double* rT = sm.psi; int* tmap = sm.itmp;
+    GR_PTR(double) dT = sm.key; GR_PTR(double) rT = sm.psi; GR_PTR(int) tmap = sm.itmp;
     if (tid < k) pv.w[tid] = trunc ? 0.0 : 1.0;
     // with the drafted tuple at hand only the system it selects is solved
     const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
@@ -925,10 +937,11 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
         lo = hi + 1;
     }
     if (status == GR_OK && skipped) status = GR_PARTIAL_RULE;
-    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
+    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b, GR_CHECK_FLAG,
+               wv.h->check);
     if (fused && status != kNeedFallback) {
         __syncthreads();                       // the rule this CTA wrote is visible to its first warp
-        fused_draw(fa, pv.h, b, n, smem_raw + L.uni * 8);
+        fused_draw(fa, pv.h, b, n, smem_raw + L.uni * 8, GR_CHECK_FLAG);
     }
 }
 

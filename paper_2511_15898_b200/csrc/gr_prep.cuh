@@ -9,7 +9,7 @@ namespace gr {
 constexpr int kNeedFallback = 100;   // internal status: the fast kernel asks the robust kernel to redo the instance
 
 // CTA-wide reductions; `scratch` needs one double per warp.  Every thread gets the result.
-__device__ inline double block_reduce_max(double v, double* scratch) {
+__device__ inline double block_reduce_max(double v, GR_PTR(double) scratch) {
     for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
     const int nw = blockDim.x >> 5;
     __syncthreads();
@@ -19,7 +19,7 @@ __device__ inline double block_reduce_max(double v, double* scratch) {
     for (int i = 1; i < nw; i++) r = fmax(r, scratch[i]);
     return r;
 }
-__device__ inline double block_reduce_sum(double v, double* scratch) {
+__device__ inline double block_reduce_sum(double v, GR_PTR(double) scratch) {
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     const int nw = blockDim.x >> 5;
     __syncthreads();
@@ -32,20 +32,23 @@ __device__ inline double block_reduce_sum(double v, double* scratch) {
 
 // shared-memory arrays of the preparation (KP entries each; psi and Dr: KP + 4)
 struct PrepSm {
-    double *d, *tg, *p, *r, *key, *psi, *Dr;
-    int *id, *blk, *itmp;
-    double* red;     // one double per warp of reduction scratch
-    double* out3;    // 3 doubles: jstar, nblocks, alpha*
+    GR_PTR(double) d, tg, p, r, key, psi, Dr;
+    GR_PTR(int) id, blk, itmp;
+    GR_PTR(double) red;     // one double per warp of reduction scratch
+    GR_PTR(double) out3;    // 3 doubles: jstar, nblocks, alpha*
 };
 struct PrepResult { int k, jstar, nblocks; double alpha_star, lse_t; };
 
-struct WsView { const WsHeader* h; const int* id; const float* dl; const float* tl; };
-__device__ inline WsView view_ws(const char* ws, long long b) {
+struct WsView { const WsHeader* h; GR_PTR(const int) id; GR_PTR(const float) dl; GR_PTR(const float) tl; };
+__device__ inline WsView view_ws(const char* ws, long long b, int* flag = nullptr) {
     WsView v;
     v.h = reinterpret_cast<const WsHeader*>(ws + (size_t)b * ws_stride());
-    v.id = reinterpret_cast<const int*>((const char*)v.h + sizeof(WsHeader));
-    v.dl = reinterpret_cast<const float*>(v.id + kMaxSupport);
-    v.tl = v.dl + kMaxSupport;
+    const int* ids = reinterpret_cast<const int*>((const char*)v.h + sizeof(WsHeader));
+    const float* dls = reinterpret_cast<const float*>(ids + kMaxSupport);
+    v.id = GR_MKPTR(const int, ids, kMaxSupport, flag);
+    v.dl = GR_MKPTR(const float, dls, kMaxSupport, flag);
+    v.tl = GR_MKPTR(const float, dls + kMaxSupport, kMaxSupport, flag);
+    (void)flag;
     return v;
 }
 
@@ -183,7 +186,8 @@ __device__ inline PrepResult prep_instance(const PrepSm& sm, const WsView& wv, H
 //   outer:  T in V \ H*,   epsilon_T = 1 - (drf(H*) + drf(T))^n  <= tau,
 // i.e. tokens in decreasing drf (equal drf: smaller id first) until the bound holds.  in_T[pos] = 1 / 0 for the
 // k support positions (ratio order); scratch: k ints.  Every thread of the CTA calls it (blockDim.x >= k).
-__device__ inline void truncation_sets(const PrepSm& sm, int* in_T, int* scratch, int k, int jstar, int n, double tau)
+__device__ inline void truncation_sets(const PrepSm& sm, GR_PTR(int) in_T, GR_PTR(int) scratch, int k, int jstar, int n,
+                                       double tau)
 {
     const int tid = threadIdx.x;
     if (tid < k) {
@@ -225,8 +229,9 @@ __device__ inline void truncation_sets(const PrepSm& sm, int* in_T, int* scratch
 
 // The T-part of positions lo .. hi-1 gathered into contiguous arrays (draft masses, right-hand sides, positions);
 // returns how many.  Every thread of the CTA calls it; `count` is one int of shared memory.
-__device__ inline int gather_truncated(const int* in_T, int lo, int hi, const double* d, const double* rhs, double* dT,
-                                       double* rT, int* map, int* count)
+__device__ inline int gather_truncated(GR_PTR(const int) in_T, int lo, int hi, GR_PTR(const double) d,
+                                       GR_PTR(const double) rhs, GR_PTR(double) dT, GR_PTR(double) rT, GR_PTR(int) map,
+                                       int* count)
 {
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -240,8 +245,11 @@ __device__ inline int gather_truncated(const int* in_T, int lo, int hi, const do
 }
 
 // Rule arrays (except w, which the solvers write as they go) and the header.
+// `check_flag` / `check_before`: the bounds-checked build's per-CTA flag and what the streaming kernel reported for
+// the row (nullptr / 0 otherwise): a skipped access turns the status into GR_CHECK_FAILED.
 __device__ inline void write_rule(const PrepSm& sm, const ParamView& pv, int KP, const PrepResult& pr, int n,
-                                  int status, double gnorm, int iters, float* alpha_out, int* status_out, long long b)
+                                  int status, double gnorm, int iters, float* alpha_out, int* status_out, long long b,
+                                  const int* check_flag = nullptr, int check_before = 0)
 {
     const int tid = threadIdx.x;
     for (int j = tid; j < KP; j += blockDim.x) {
@@ -254,6 +262,7 @@ __device__ inline void write_rule(const PrepSm& sm, const ParamView& pv, int KP,
     }
     __syncthreads();
     if (tid == 0) {
+        if (check_before || (check_flag && *check_flag)) status = GR_CHECK_FAILED;
         Header* h = pv.h;
         h->n = n; h->k = pr.k; h->jstar = pr.jstar; h->nblocks = pr.nblocks; h->status = status;
         h->alpha_star = pr.alpha_star;

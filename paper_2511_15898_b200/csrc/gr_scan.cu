@@ -78,7 +78,7 @@ __device__ __forceinline__ void osm_warp_reduce(float& m, float& s, float sc) {
 }
 
 struct CandList {
-    float* v; int* id; int* cnt;
+    GR_PTR(float) v; GR_PTR(int) id; int* cnt;
 };
 // every lane of the warp calls this; `ok` marks lanes holding a real element
 __device__ __forceinline__ void push_one(const CandList& cl, float val, int id, bool ok, float tau, int lane) {
@@ -118,7 +118,7 @@ __device__ __forceinline__ void push_lane(const CandList& cl, float val, int id,
 // Exact selection of the ksel largest composite keys of the draft row by eight 8-bit
 // radix passes over the row (slow path, taken only when the candidate list overflowed).
 template <typename T>
-__device__ void exact_select_slow(const T* prow, int V, int ksel, const CandList& cl, int* hist /*256 ints*/,
+__device__ void exact_select_slow(const T* prow, int V, int ksel, const CandList& cl, GR_PTR(int) hist /*256 ints*/,
                                   unsigned long long* s_prefix, int* s_need) {
     const int tid = threadIdx.x;
     if (tid == 0) { *s_prefix = 0ull; *s_need = ksel; }
@@ -172,10 +172,15 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
     constexpr int NB = S / U;
     static_assert(S % U == 0, "chunk must be a whole number of batches");
 
-    __shared__ unsigned long long s_keys[kCandCap];
-    __shared__ float2 s_chunk[kMaxChunks];
+    __shared__ unsigned long long s_keys_raw[kCandCap];
+    __shared__ float2 s_chunk_raw[kMaxChunks];
     __shared__ float s_dm[kScanWarps], s_ds[kScanWarps];
-    __shared__ int s_hist[256];
+    __shared__ int s_hist_raw[256];
+    GR_CHECK_FLAG_DECL;
+    GR_CHECK_FLAG_INIT;
+    GR_PTR(unsigned long long) s_keys = GR_MKPTR(unsigned long long, s_keys_raw, kCandCap, GR_CHECK_FLAG);
+    GR_PTR(float2) s_chunk = GR_MKPTR(float2, s_chunk_raw, kMaxChunks, GR_CHECK_FLAG);
+    GR_PTR(int) s_hist = GR_MKPTR(int, s_hist_raw, 256, GR_CHECK_FLAG);
     __shared__ unsigned long long s_prefix;
     __shared__ int s_need, s_cnt, s_bad;
     __shared__ float s_tau;
@@ -191,8 +196,8 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
     const int tail = V - vec_end;
 
     CandList cl;
-    cl.v = reinterpret_cast<float*>(s_keys);
-    cl.id = reinterpret_cast<int*>(s_keys) + kCandCap;
+    cl.v = GR_MKPTR(float, reinterpret_cast<float*>(s_keys_raw), kCandCap, GR_CHECK_FLAG);
+    cl.id = GR_MKPTR(int, reinterpret_cast<int*>(s_keys_raw) + kCandCap, kCandCap, GR_CHECK_FLAG);
     cl.cnt = &s_cnt;
     const bool take_all = !kFull && (V <= kCandCap);       // every element is a candidate
     const bool use_tau = !kFull && !take_all;
@@ -234,6 +239,9 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
             for (int u = 0; u < U; u++) {
                 idx[u] = head + c * kChunk + ((nb * U + u) * 32 + lane) * N;
                 ok[u] = cvalid && (idx[u] + N <= vec_end);
+#ifdef GR_CHECK
+                if (ok[u] && (idx[u] < 0 || idx[u] + N > V || ((size_t)(qrow + idx[u]) & 15))) { s_check_flag = 1; ok[u] = false; }
+#endif
                 if (ok[u]) {
                     qv[u] = __ldcs(reinterpret_cast<const typename VT::Vec*>(qrow + idx[u]));
                     pv[u] = __ldcs(reinterpret_cast<const typename VT::Vec*>(prow + idx[u]));
@@ -358,9 +366,11 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
         }
         __syncthreads();
         char* wsb = ws + (size_t)b * ws_stride();
-        int* w_id = reinterpret_cast<int*>(wsb + sizeof(WsHeader));
-        float* w_dl = reinterpret_cast<float*>(w_id + kMaxSupport);
-        float* w_tl = w_dl + kMaxSupport;
+        int* w_id_raw = reinterpret_cast<int*>(wsb + sizeof(WsHeader));
+        float* w_dl_raw = reinterpret_cast<float*>(w_id_raw + kMaxSupport);
+        GR_PTR(int) w_id = GR_MKPTR(int, w_id_raw, kMaxSupport, GR_CHECK_FLAG);
+        GR_PTR(float) w_dl = GR_MKPTR(float, w_dl_raw, kMaxSupport, GR_CHECK_FLAG);
+        GR_PTR(float) w_tl = GR_MKPTR(float, w_dl_raw + kMaxSupport, kMaxSupport, GR_CHECK_FLAG);
         if (M < nsel) nsel = M;   // cannot happen for finite rows; keeps the writes in range
 #pragma unroll
         for (int u = 0; u < kPer; u++) {
@@ -372,6 +382,9 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
                 if (rank < nsel) {
                     w_id[rank] = ii[u];
                     w_dl[rank] = vv[u];
+#ifdef GR_CHECK
+                    if (ii[u] < 0 || ii[u] >= V) { s_check_flag = 1; ii[u] = 0; }
+#endif
                     w_tl[rank] = load_logit<T>(qrow, ii[u]);
                 }
             }
@@ -380,17 +393,24 @@ scan_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int ksel, f
 
     // ---- outputs: workspace header, chunk table and the header fields owned by this kernel
     // (params == nullptr: the caller wants the workspace record only)
+    char* pb = params ? params + (size_t)b * pstride : nullptr;
+    if (pb) {
+        ParamView pv = view_params(pb, kcap, V, GR_CHECK_FLAG);
+        for (int c = tid; c < nch; c += kScanThreads) pv.chunk[c] = s_chunk[c];
+    }
+#ifdef GR_CHECK
+    __syncthreads();
+#endif
     if (tid == 0) {
         WsHeader* wh = reinterpret_cast<WsHeader*>(ws + (size_t)b * ws_stride());
         wh->lse_t = s_lse[0];
         wh->lse_d = s_lse[1];
         wh->count = nsel;
         wh->bad = s_bad;
+        wh->check = GR_CHECK_VALUE;
     }
     if (params == nullptr) return;
-    char* pb = params + (size_t)b * pstride;
-    ParamView pv = view_params(pb, kcap);
-    for (int c = tid; c < nch; c += kScanThreads) pv.chunk[c] = s_chunk[c];
+    ParamView pv = view_params(pb, kcap, V, GR_CHECK_FLAG);
     if (tid == 0) {
         Header* h = pv.h;
         h->magic = 0;            // completed by the solve kernel

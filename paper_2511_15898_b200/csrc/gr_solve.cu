@@ -68,9 +68,9 @@ __host__ int solve_pick_tile(int KP, int n, int max_bytes) {
 __host__ int solve_smem_bytes(int KP, int n, int Qt) { return SolveLayout(KP, n, Qt).total_bytes; }
 
 struct Sm {
-    double *d, *tg, *p, *r, *key, *w, *psi, *Dr, *alpha, *alpha_prev, *delta, *g, *g2, *col, *E, *J, *tq, *cq, *X, *H,
-        *A, *P, *PP, *PX, *AX, *gq, *g2q, *scal;
-    int *id, *blk, *order, *itmp;
+    GR_PTR(double) d, tg, p, r, key, w, psi, Dr, alpha, alpha_prev, delta, g, g2, col, E, J, tq, cq, X, H, A, P, PP, PX, AX,
+        gq, g2q, scal;
+    GR_PTR(int) id, blk, order, itmp;
     int KP, n, Qt;
 };
 
@@ -82,11 +82,12 @@ enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SH
 // Evaluate g (and, if want_jac, the packed lower triangle of the Hessian) at sm.alpha[0..m).
 // d = draft masses of the system's tokens, hmass = draft mass of everything of higher ratio
 // (outer blocks), slack = 1 for the inner system.  Returns the number of quadrature nodes.
-__device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, int slack, bool want_jac, double qstep)
+__device__ int eval_system(const Sm& sm, int m, GR_PTR(const double) d, double hmass, int slack, bool want_jac,
+                           double qstep)
 {
     const int tid = threadIdx.x;
     const int n = sm.n, n1 = sm.n + 1, KP = sm.KP, Qt = sm.Qt;
-    double* red = sm.scal + 16;
+    GR_PTR(double) red = sm.scal + 16;
     // weights and their range
     double wj = 0.0;
     if (tid < m) { wj = exp(sm.alpha[tid]); sm.w[tid] = wj; sm.g[tid] = 0.0; sm.g2[tid] = 0.0; }
@@ -123,7 +124,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             const int q = task / m, j = task - q * m;
             const double x = exp(-sm.tq[q] * sm.w[j]);
             sm.X[q * KP + j] = x;
-            double* Hq = sm.H + (size_t)q * n1 * KP;
+            GR_PTR(double) Hq = sm.H + (size_t)q * n1 * KP;
             for (int c = 1; c <= n; c++) {
                 double acc = 0.0;
                 for (int a = 1; a < c; a++) acc += sm.E[a * KP + j] * Hq[(c - a) * KP + j];
@@ -133,7 +134,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
         // partial products of the factors f_j over token groups
         for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
             const int q = task / kGroups, grp = task - q * kGroups;
-            double* PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+            GR_PTR(double) PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
             if (grp == 0) {
                 double hp = 1.0, fc = 1.0;
                 for (int c = 0; c <= n; c++) { PPq[c] = hp / fc; hp *= hmass; fc *= (double)(c + 1); }
@@ -145,7 +146,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
         __syncthreads();
         for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
             const int q = task / kGroups, grp = task - q * kGroups;
-            double* PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+            GR_PTR(double) PPq = sm.PP + (size_t)(q * kGroups + grp) * n1;
             const int j0 = grp * gsz, j1 = min(m, j0 + gsz);
             for (int j = j0; j < j1; j++) {
                 if (j == da || j == db) continue;          // dominant factors are applied after the tree
@@ -162,8 +163,8 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             for (int task = tid; task < qn * kGroups; task += kSolveThreads) {
                 const int q = task / kGroups, grp = task - q * kGroups;
                 if ((grp % (2 * stride)) == 0 && grp + stride < kGroups) {
-                    double* Aq = sm.PP + (size_t)(q * kGroups + grp) * n1;
-                    const double* Bq = sm.PP + (size_t)(q * kGroups + grp + stride) * n1;
+                    GR_PTR(double) Aq = sm.PP + (size_t)(q * kGroups + grp) * n1;
+                    GR_PTR(const double) Bq = sm.PP + (size_t)(q * kGroups + grp + stride) * n1;
                     for (int c = n; c >= 0; c--) {
                         double acc = 0.0;
                         for (int a = 0; a <= c; a++) acc += Aq[a] * Bq[c - a];
@@ -178,8 +179,8 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             // PX[q][2] = full product.
             for (int task = tid; task < qn * 3; task += kSolveThreads) {
                 const int q = task / 3, which = task - q * 3;
-                const double* Lab = sm.PP + (size_t)(q * kGroups) * n1;
-                double* out = sm.PX + (size_t)(q * 3 + which) * n1;
+                GR_PTR(const double) Lab = sm.PP + (size_t)(q * kGroups) * n1;
+                GR_PTR(double) out = sm.PX + (size_t)(q * 3 + which) * n1;
                 for (int c = 0; c <= n; c++) out[c] = Lab[c];
                 // factors to apply: which 0 -> f_b, which 1 -> f_a, which 2 -> f_a and f_b
                 for (int pass = 0; pass < 2; pass++) {
@@ -198,11 +199,11 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
         // per (node, token): gradient integrand; series A = P h scaled for the Hessian
         for (int task = tid; task < qn * m; task += kSolveThreads) {
             const int q = task / m, j = task - q * m;
-            const double* Pq = da >= 0 ? sm.PX + (size_t)(q * 3 + 2) * n1 : sm.PP + (size_t)(q * kGroups) * n1;
-            double* Hq = sm.H + (size_t)q * n1 * KP;
+            GR_PTR(const double) Pq = da >= 0 ? sm.PX + (size_t)(q * 3 + 2) * n1 : sm.PP + (size_t)(q * kGroups) * n1;
+            GR_PTR(double) Hq = sm.H + (size_t)q * n1 * KP;
             if (j == da || j == db) {
                 // dominant token: dM/dx_j = n! [lambda^n] e_j L_j with L_j the product of all other factors
-                const double* Lj = sm.PX + (size_t)(q * 3 + (j == da ? 0 : 1)) * n1;
+                GR_PTR(const double) Lj = sm.PX + (size_t)(q * 3 + (j == da ? 0 : 1)) * n1;
                 double val = 0.0;
                 for (int c = 1; c <= n; c++) val += Lj[n - c] * sm.E[c * KP + j];
                 const double u = sm.w[j] * sm.X[q * KP + j];
@@ -211,7 +212,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
                 sm.gq[q * KP + j] = gi;
                 sm.g2q[q * KP + j] = gi * sm.tq[q] * sm.w[j];
                 if (want_jac) {
-                    double* Aq = sm.A + (size_t)q * n1 * KP;
+                    GR_PTR(double) Aq = sm.A + (size_t)q * n1 * KP;
                     const double sa = cg * sm.tq[q] * u;
                     for (int e = 1; e < n; e++) {
                         double acc = 0.0;
@@ -220,8 +221,8 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
                     }
                     if (j == da && db >= 0) {
                         // for the pair (a, b): the series e_a times the product without both
-                        const double* Lab = sm.PP + (size_t)(q * kGroups) * n1;
-                        double* Ax = sm.AX + (size_t)q * n1;
+                        GR_PTR(const double) Lab = sm.PP + (size_t)(q * kGroups) * n1;
+                        GR_PTR(double) Ax = sm.AX + (size_t)q * n1;
                         for (int e = 1; e < n; e++) {
                             double acc = 0.0;
                             for (int c = 1; c <= e; c++) acc += sm.E[c * KP + j] * Lab[e - c];
@@ -240,7 +241,7 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
             sm.gq[q * KP + j] = gi;
             sm.g2q[q * KP + j] = gi * sm.tq[q] * sm.w[j];
             if (want_jac) {
-                double* Aq = sm.A + (size_t)q * n1 * KP;
+                GR_PTR(double) Aq = sm.A + (size_t)q * n1 * KP;
                 const double sa = cg * sm.tq[q] * u;
                 for (int e = 1; e < n; e++) {
                     double acc = 0.0;
@@ -266,10 +267,10 @@ __device__ int eval_system(const Sm& sm, int m, const double* d, double hmass, i
                     // tokens pair through the product without both
                     const int ia = (doml && !domi) ? l : i, ih = (doml && !domi) ? i : l;
                     for (int q = 0; q < qn; q++) {
-                        const double* Aq = sm.A + (size_t)q * n1 * KP;
-                        const double* Hq = sm.H + (size_t)q * n1 * KP;
+                        const GR_PTR(double) Aq = sm.A + (size_t)q * n1 * KP;
+                        const GR_PTR(double) Hq = sm.H + (size_t)q * n1 * KP;
                         if (domi && doml) {
-                            const double* Ax = sm.AX + (size_t)q * n1;
+                            const GR_PTR(double) Ax = sm.AX + (size_t)q * n1;
                             for (int c = 1; c < n; c++) acc += Ax[n - c] * Hq[c * KP + db];
                         } else {
                             for (int c = 1; c < n; c++) acc += Aq[(n - c) * KP + ia] * Hq[c * KP + ih];
@@ -333,11 +334,11 @@ __device__ void chol_solve(const Sm& sm, int m)
 
 // Newton iteration for one system.  On return sm.w[0..m) holds exp(alpha).
 // Returns the status; *gnorm and *iters receive the final L1 gradient norm and the evaluations spent.
-__device__ int solve_system(const Sm& sm, int m, const double* d, const double* rhs, double hmass, int slack,
-                            double tol, int max_iters, double qstep, double* gnorm, int* iters)
+__device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(const double) rhs, double hmass,
+                            int slack, double tol, int max_iters, double qstep, double* gnorm, int* iters)
 {
     const int tid = threadIdx.x, n = sm.n, KP = sm.KP;
-    double* red = sm.scal + 16;
+    GR_PTR(double) red = sm.scal + 16;
     // E[c][j] = d_j^c / c!
     if (tid < m) {
         double pw = 1.0, fc = 1.0;
@@ -449,12 +450,14 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ int s_sel;
+    GR_CHECK_FLAG_DECL;
+    GR_CHECK_FLAG_INIT;
     const bool fused = fa.draft != nullptr;
     const int tid = threadIdx.x;
     const long long b = blockIdx.x;
     char* pb = params + (size_t)b * pstride;
-    ParamView pv = view_params(pb, kcap);
-    const WsView wv = view_ws(ws, b);
+    ParamView pv = view_params(pb, kcap, V, GR_CHECK_FLAG);
+    const WsView wv = view_ws(ws, b, GR_CHECK_FLAG);
     // second pass after the fast kernel: only the instances it flagged are redone
     if (only_flagged && !(pv.h->magic == kMagic && pv.h->status == kNeedFallback)) return;
     if (kcap == 0 || wv.h->bad != 0 || wv.h->count <= 0) {
@@ -462,7 +465,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
         if (tid == 0) write_no_rule(pv.h, n, wv.h->bad != 0, alpha_out, status_out, b);
         if (fused) {
             __syncthreads();
-            fused_draw(fa, pv.h, b, n, smem_raw);
+            fused_draw(fa, pv.h, b, n, smem_raw, GR_CHECK_FLAG);
         }
         return;
     }
@@ -471,17 +474,29 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     SolveLayout L(KP, n, Qt);
     double* base = reinterpret_cast<double*>(smem_raw);
     Sm sm;
-    sm.d = base + L.d; sm.tg = base + L.tg; sm.p = base + L.p; sm.r = base + L.r; sm.key = base + L.key;
-    sm.w = base + L.w; sm.psi = base + L.psi; sm.Dr = base + L.Dr; sm.alpha = base + L.alpha;
-    sm.alpha_prev = base + L.alpha_prev; sm.delta = base + L.delta; sm.g = base + L.g; sm.g2 = base + L.g2;
-    sm.col = base + L.col; sm.E = base + L.E; sm.J = base + L.J; sm.tq = base + L.tq; sm.cq = base + L.cq;
-    sm.X = base + L.X; sm.H = base + L.H; sm.A = base + L.A; sm.P = base + L.P; sm.PP = base + L.PP;
-    sm.PX = base + L.PX; sm.AX = base + L.AX;
-    sm.gq = base + L.gq; sm.g2q = base + L.g2q; sm.scal = base + L.scal;
+    int* const ck = GR_CHECK_FLAG;
+    (void)ck;
+    const int n1c = n + 1;
+    sm.d = GR_MKPTR(double, base + L.d, KP, ck); sm.tg = GR_MKPTR(double, base + L.tg, KP, ck);
+    sm.p = GR_MKPTR(double, base + L.p, KP, ck); sm.r = GR_MKPTR(double, base + L.r, KP, ck);
+    sm.key = GR_MKPTR(double, base + L.key, KP, ck); sm.w = GR_MKPTR(double, base + L.w, KP, ck);
+    sm.psi = GR_MKPTR(double, base + L.psi, KP + 4, ck); sm.Dr = GR_MKPTR(double, base + L.Dr, KP + 4, ck);
+    sm.alpha = GR_MKPTR(double, base + L.alpha, KP, ck); sm.alpha_prev = GR_MKPTR(double, base + L.alpha_prev, KP, ck);
+    sm.delta = GR_MKPTR(double, base + L.delta, KP, ck); sm.g = GR_MKPTR(double, base + L.g, KP, ck);
+    sm.g2 = GR_MKPTR(double, base + L.g2, KP, ck); sm.col = GR_MKPTR(double, base + L.col, KP, ck);
+    sm.E = GR_MKPTR(double, base + L.E, KP * n1c, ck); sm.J = GR_MKPTR(double, base + L.J, KP * (KP + 1) / 2, ck);
+    sm.tq = GR_MKPTR(double, base + L.tq, Qt, ck); sm.cq = GR_MKPTR(double, base + L.cq, Qt, ck);
+    sm.X = GR_MKPTR(double, base + L.X, Qt * KP, ck); sm.H = GR_MKPTR(double, base + L.H, Qt * n1c * KP, ck);
+    sm.A = GR_MKPTR(double, base + L.A, Qt * n1c * KP, ck); sm.P = GR_MKPTR(double, base + L.P, Qt * n1c, ck);
+    sm.PP = GR_MKPTR(double, base + L.PP, Qt * kGroups * n1c, ck); sm.PX = GR_MKPTR(double, base + L.PX, Qt * 3 * n1c, ck);
+    sm.AX = GR_MKPTR(double, base + L.AX, Qt * n1c, ck);
+    sm.gq = GR_MKPTR(double, base + L.gq, Qt * KP, ck); sm.g2q = GR_MKPTR(double, base + L.g2q, Qt * KP, ck);
+    sm.scal = GR_MKPTR(double, base + L.scal, 32, ck);
     int* ib = reinterpret_cast<int*>(smem_raw + L.ints);
-    sm.id = ib; sm.blk = ib + KP; sm.order = ib + 2 * KP; sm.itmp = ib + 3 * KP;
+    sm.id = GR_MKPTR(int, ib, KP, ck); sm.blk = GR_MKPTR(int, ib + KP, KP, ck);
+    sm.order = GR_MKPTR(int, ib + 2 * KP, KP, ck); sm.itmp = GR_MKPTR(int, ib + 3 * KP, KP, ck);
     sm.KP = KP; sm.n = n; sm.Qt = Qt;
-    double* red = sm.scal + 16;
+    GR_PTR(double) red = sm.scal + 16;
 
     PrepSm ps;
     ps.d = sm.d; ps.tg = sm.tg; ps.p = sm.p; ps.r = sm.r; ps.key = sm.key; ps.psi = sm.psi; ps.Dr = sm.Dr;
@@ -500,7 +515,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
         truncation_sets(ps, sm.order, sm.itmp, k, jstar, n, tau);
         tol = 5.0 * tau;
     }
-    double* dT = sm.key; double* rT = sm.psi; int* tmap = sm.itmp;
+    GR_PTR(double) dT = sm.key; GR_PTR(double) rT = sm.psi; GR_PTR(int) tmap = sm.itmp;
     if (tid < k) pv.w[tid] = trunc ? 0.0 : 1.0;
     // with the drafted tuple at hand only the system it selects is solved
     const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
@@ -563,10 +578,11 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     }
 
     if (status == GR_OK && skipped) status = GR_PARTIAL_RULE;
-    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b);
+    write_rule(ps, pv, KP, pr, n, status, gnorm_total, iters_total, alpha_out, status_out, b, GR_CHECK_FLAG,
+               wv.h->check);
     if (fused) {
         __syncthreads();                       // the rule this CTA wrote is visible to its first warp
-        fused_draw(fa, pv.h, b, n, smem_raw);
+        fused_draw(fa, pv.h, b, n, smem_raw, GR_CHECK_FLAG);
     }
 }
 

@@ -10,6 +10,8 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
               int* __restrict__ out_token, unsigned char* __restrict__ out_acc, int* __restrict__ status_out)
 {
     __shared__ double s_scratch[kVerifyWarps][kVerifyScratchBytes / 8];
+    GR_CHECK_FLAG_DECL;
+    GR_CHECK_FLAG_INIT;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     const int b = blockIdx.x * kVerifyWarps + wib;
     if (b >= batch) return;
@@ -23,8 +25,10 @@ verify_kernel(const char* __restrict__ params, const int* __restrict__ draft, co
         if (h->magic != kMagic) status = GR_STALE_PARAMS;
     }
     if (status == GR_OK)
-        verify_instance(h, draft + (size_t)b * h->n, uni + 2 * (size_t)b, lane, verify_scratch(s_scratch[wib]), false,
-                        token, accepted, status);
+        verify_instance(h, draft + (size_t)b * h->n, uni + 2 * (size_t)b, lane,
+                        verify_scratch(s_scratch[wib], GR_CHECK_FLAG), false, token, accepted, status);
+    __syncwarp();
+    if (GR_CHECK_VALUE) status = GR_CHECK_FAILED;      // (the flag is shared by the CTA's four instances)
     if (lane == 0) {
         out_token[b] = token;
         out_acc[b] = (unsigned char)accepted;
@@ -57,7 +61,7 @@ read_slice_kernel(const char* __restrict__ params, const int* __restrict__ draft
         n = h->n < nmax ? h->n : nmax;
         status = h->status;
         if (status == GR_OK || status == GR_NOT_CONVERGED) {
-            ParamView pv = view_params((void*)h, h->kcap);
+            ParamView pv = view_params((void*)h, h->kcap, h->V, nullptr);
             tok = lane < h->n ? draft[(size_t)b * h->n + lane] : -1;
             const int rs = h->k > 0 ? slice_instance(h, pv, tok, lane, sl) : GR_SUPPORT_TOO_LARGE;
             if (rs != GR_OK) { status = rs; sl.uniq = false; sl.pi = 0.0; sl.rho = 0.0; }

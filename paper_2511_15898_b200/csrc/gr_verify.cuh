@@ -18,15 +18,20 @@ struct FusedArgs {
 
 // Shared-memory scratch of one verifying warp.
 struct VerifyScratch {
-    int* l_id; double* l_r; int* s_id; double* s_p;       // kMaxSupport entries each
+    GR_PTR(int) l_id; GR_PTR(double) l_r; GR_PTR(int) s_id; GR_PTR(double) s_p;       // kMaxSupport entries each
+    int* flag;                                              // bounds-checked build: where skipped accesses are reported
 };
 constexpr int kVerifyScratchBytes = kMaxSupport * 24;
-__device__ inline VerifyScratch verify_scratch(void* base) {     // base: 8-byte aligned, kVerifyScratchBytes long
+// base: 8-byte aligned, kVerifyScratchBytes long
+__device__ inline VerifyScratch verify_scratch(void* base, int* flag = nullptr) {
     VerifyScratch v;
-    v.l_r = reinterpret_cast<double*>(base);
-    v.s_p = v.l_r + kMaxSupport;
-    v.l_id = reinterpret_cast<int*>(v.s_p + kMaxSupport);
-    v.s_id = v.l_id + kMaxSupport;
+    double* lr = reinterpret_cast<double*>(base);
+    int* li = reinterpret_cast<int*>(lr + 2 * kMaxSupport);
+    v.l_r = GR_MKPTR(double, lr, kMaxSupport, flag);
+    v.s_p = GR_MKPTR(double, lr + kMaxSupport, kMaxSupport, flag);
+    v.l_id = GR_MKPTR(int, li, kMaxSupport, flag);
+    v.s_id = GR_MKPTR(int, li + kMaxSupport, kMaxSupport, flag);
+    v.flag = flag;
     return v;
 }
 
@@ -47,7 +52,7 @@ __device__ __forceinline__ double warp_incl_scan(double v, int lane) {
 // Two levels: per-chunk masses from the scan kernel's table minus the flow p_i of the
 // support ids in the chunk, then an exact fp64 pass over the one chunk selected.
 __device__ inline int resample_draw(const Header* h, const ParamView& pv, int k, double frac, int lane,
-                             int* l_id, double* l_r, int* s_id, double* s_p)
+                             GR_PTR(int) l_id, GR_PTR(double) l_r, GR_PTR(int) s_id, GR_PTR(double) s_p)
 {
     const int nch = h->nch, head = h->head, V = h->V, dtype = h->dtype;
     const double T = (double)h->temp_target, lse = h->lse_t;
@@ -197,7 +202,7 @@ __device__ inline void verify_instance(const Header* h, const int* draft_row, co
         if (!allow_partial) return;
         status = GR_OK;
     }
-    ParamView pv = view_params((void*)h, h->kcap);
+    ParamView pv = view_params((void*)h, h->kcap, h->V, vs.flag);
     const int n = h->n, k = h->k;
     const double u0 = (double)uni_row[0], u1 = (double)uni_row[1];
     const int tok = lane < n ? draft_row[lane] : -1;
@@ -230,8 +235,8 @@ __device__ inline void verify_instance(const Header* h, const int* draft_row, co
 // Which system the drafted tuple selects (Eq. "cases"): -1 the inner system (every drafted token in H*), b >= 0 the
 // outer block b (the lowest-ratio block met), -2 when a drafted token is outside the support (then every system is
 // solved and the draw reports the error).  Every thread of the CTA calls it; id / blk are in ratio order.
-__device__ inline int selected_system(const int* draft_row, int n, int k, int jstar, const int* sid, const int* sblk,
-                                      int* s_sel)
+__device__ inline int selected_system(const int* draft_row, int n, int k, int jstar, GR_PTR(const int) sid,
+                                      GR_PTR(const int) sblk, int* s_sel)
 {
     const int tid = threadIdx.x;
     if (tid == 0) *s_sel = -1;
@@ -252,13 +257,15 @@ __device__ inline int selected_system(const int* draft_row, int n, int k, int js
 
 // Draw of instance b by warp 0 of a solve kernel's CTA, after the rule (or the no-rule header) was written and the
 // CTA synchronised.
-__device__ inline void fused_draw(const FusedArgs& fa, const Header* h, long long b, int n, void* scratch)
+__device__ inline void fused_draw(const FusedArgs& fa, const Header* h, long long b, int n, void* scratch,
+                                  int* check_flag = nullptr)
 {
     if (threadIdx.x >= 32) return;
     const int lane = threadIdx.x;
     int token, accepted, status;
-    verify_instance(h, fa.draft + (size_t)b * n, fa.uni + 2 * (size_t)b, lane, verify_scratch(scratch), true, token,
-                    accepted, status);
+    verify_instance(h, fa.draft + (size_t)b * n, fa.uni + 2 * (size_t)b, lane, verify_scratch(scratch, check_flag), true,
+                    token, accepted, status);
+    if (check_flag && *check_flag) status = GR_CHECK_FAILED;
     if (lane == 0) {
         fa.out_token[b] = token;
         fa.out_acc[b] = (unsigned char)accepted;
