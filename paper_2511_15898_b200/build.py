@@ -71,7 +71,7 @@ def build_library(force: bool = False, verbose: bool = False, check: bool = Fals
     if failed:
         raise RuntimeError("nvcc failed:\n" + "\n".join(failed))
     res = subprocess.run([_nvcc(), "-shared", "-cudart", "static", "-gencode", "arch=compute_100a,code=sm_100a"]
-                         + objs + ["-o", LIB], capture_output=True, text=True)
+                         + objs + ["-ldl", "-o", LIB], capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     return LIB

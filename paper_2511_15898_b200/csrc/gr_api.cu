@@ -86,10 +86,15 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
     const int kfull = su.kfull, kcap = su.kcap, pstride = su.pstride;
     const bool full_large = kcap == 0;
     cudaStream_t st = (cudaStream_t)stream;
-    gr::launch_scan(q_logits, p_logits, dtype, V, kfull, full_large, (double)temp_target, (double)temp_draft, batch,
-                    (char*)workspace, (char*)params, pstride, kcap, st);
+    gr::NvtxRange whole(fa.draft ? "gr_solve_verify" : "gr_solve");
+    {
+        gr::NvtxRange r("gr:scan");
+        gr::launch_scan(q_logits, p_logits, dtype, V, kfull, full_large, (double)temp_target, (double)temp_draft,
+                        batch, (char*)workspace, (char*)params, pstride, kcap, st);
+    }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     if (scan_done && cudaEventRecord(scan_done, st) != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+    gr::NvtxRange r(fa.draft ? "gr:solve+draw" : "gr:solve");
     int rc = gr::launch_solve_any((const char*)workspace, (char*)params, pstride, kcap, V, n, topk,
                                   (double)temp_target, (double)temp_draft, tol, max_iters, qstep, tau, batch,
                                   force_robust, alpha_star, status, fa, st);
@@ -143,6 +148,7 @@ int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, 
     const int kcap = gr::kcap_of(V, topk);
     if (kcap == 0) return GR_E_TOO_LARGE;
     cudaStream_t st = (cudaStream_t)stream;
+    gr::NvtxRange whole("gr_alpha_star");
     gr::launch_scan(q_logits, p_logits, dtype, V, kfull, false, (double)temp_target, (double)temp_draft, batch,
                     (char*)workspace, nullptr, 0, kcap, st);
     gr::launch_alpha((const char*)workspace, V, topk, (double)temp_target, (double)temp_draft, n_list, n_count, batch,
@@ -158,6 +164,7 @@ int gr_verify(const void* params, const int* draft_tokens, const float* uniforms
     if (batch == 0) return GR_OK;
     if (!params || !draft_tokens || !uniforms || !out_token || !out_accepted || !status) return GR_E_NULL;
     if ((uintptr_t)params & 15) return GR_E_ALIGN;
+    gr::NvtxRange whole("gr_verify");
     gr::launch_verify((const char*)params, draft_tokens, uniforms, batch, out_token, out_accepted, status,
                       (cudaStream_t)stream);
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }

@@ -1,9 +1,19 @@
 // Host-side declarations shared by the translation units that implement the C interface: the kernel launchers and
 // the argument checks common to gr_solve, gr_solve_verify and gr_solve_static.
 #pragma once
+#include <nvtx3/nvToolsExt.h>
 #include "gr_verify.cuh"
 
 namespace gr {
+
+// A named range on a profiler's timeline around the host code that enqueues one phase of the path (scan, solve,
+// verify ...).  Without a profiler attached the two calls do nothing.
+struct NvtxRange {
+    explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+    ~NvtxRange() { nvtxRangePop(); }
+    NvtxRange(const NvtxRange&) = delete;
+    NvtxRange& operator=(const NvtxRange&) = delete;
+};
 
 void launch_scan(const void* q, const void* p, int dtype, int V, int ksel, bool full_large, double temp_t,
                  double temp_d, int batch, char* ws, char* params, int pstride, int kcap, cudaStream_t st);

@@ -52,6 +52,7 @@ extern "C" int gr_solve_static(const void* q_logits, const void* p_logits, int d
     if (rs != GR_OK) return rs;
     const int pstride = su.pstride;
     cudaStream_t st = (cudaStream_t)stream;
+    gr::NvtxRange whole("gr_solve_static");
     // the streaming kernel writes every workspace field the solve kernel reads, so nothing has to be cleared
     gr::launch_scan(q_logits, p_logits, dtype, V, kfull, full_large, (double)temp_target, (double)temp_draft, batch,
                     ws, (char*)params, pstride, kcap, st);
