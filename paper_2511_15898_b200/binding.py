@@ -34,7 +34,7 @@ class Options(C.Structure):
     _fields_ = [("tol", C.c_double), ("max_iters", C.c_int), ("quad_step", C.c_double),
                 ("scan_done_event", C.c_void_p), ("force_robust", C.c_int), ("tau", C.c_double)]
 
-    def __init__(self, tol: float = 1e-9, max_iters: int = 40, quad_step: float = 0.4, scan_done_event=None,
+    def __init__(self, tol: float = 3e-7, max_iters: int = 40, quad_step: float = 0.4, scan_done_event=None,
                  force_robust: int = 0, tau: float = 0.0):
         super().__init__(tol, max_iters, quad_step, scan_done_event, force_robust, tau)
 

@@ -30,7 +30,7 @@ int check_solve_args(const void* q_logits, const void* p_logits, int dtype, int 
     if (dtype != GR_F32 && dtype != GR_BF16) return GR_E_INVALID;
     if (!(temp_target > 0.f) || !(temp_draft > 0.f) || !isfinite(temp_target) || !isfinite(temp_draft))
         return GR_E_INVALID;
-    out->tol = 1e-9; out->qstep = 0.4; out->max_iters = 40; out->tau = 0.0;
+    out->tol = 3e-7; out->qstep = 0.4; out->max_iters = 40; out->tau = 0.0;
     out->scan_done = nullptr; out->force_robust = 0;
     if (opt) {
         out->scan_done = (cudaEvent_t)opt->scan_done_event;
