@@ -88,7 +88,9 @@ extern "C" {
  *              time the two separately; NULL records nothing.      default NULL
  *   force_robust  non-zero sends every shape to the general (slower) solve kernel;
  *              by default supports of at most 128 tokens with n <= 16 take a faster
- *              kernel that computes the same rule.                  default 0
+ *              kernel that computes the same rule.  For an untruncated draft on a
+ *              vocabulary beyond GR_MAX_SUPPORT (optimal acceptance only) it selects the
+ *              whole-row sort instead of the bucketed search.         default 0
  *   tau        error threshold of Algorithm 1 (Sec. 6.2 "tunable errors", Sec. 6.3).  0 solves the
  *              convex programs on the whole support (the default: both tunable errors are 0 and `tol`
  *              is the stopping rule).  tau in (0, 1] selects the truncated variant: the inner system

@@ -100,10 +100,11 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
                                   force_robust, alpha_star, status, fa, st);
     if (rc != GR_OK) return rc;
     if (full_large) {
-        // no rule is solved for this shape, but the optimal acceptance still is (sort + prefix scan)
+        // no rule is solved for this shape, but the optimal acceptance still is (bucketed search for the minimum of
+        // psi, or with force_robust a sort of the whole row and a prefix scan)
         char* scratch = (char*)workspace + (size_t)gr::ws_stride() * (size_t)batch;
         gr::launch_fullsort(q_logits, p_logits, dtype, V, n, (double)temp_target, (double)temp_draft, batch,
-                            (const char*)workspace, scratch, (char*)params, pstride, alpha_star, st);
+                            (const char*)workspace, scratch, (char*)params, pstride, force_robust, alpha_star, st);
     }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;

@@ -297,6 +297,47 @@ def test_config4_whole_vocabulary_cells_alpha_star(n, sigma):
     assert bool((ver.token >= 0).all())
 
 
+def _alpha_both_ways(wl):
+    """alpha* of a whole-vocabulary instance by the bucketed search (default) and by the whole-row sort
+    (force_robust), and the oracle's."""
+    from oracle import gr_oracle as O
+    a = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft)
+    b = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft, G.Options(force_robust=1))
+    torch.cuda.synchronize()
+    tl = W.logits_to_f64(wl.q_logits); dl = W.logits_to_f64(wl.p_logits)
+    want = np.array([O.alpha_star_only(tl[i], dl[i], wl.n, wl.topk, wl.temp_target, wl.temp_draft)[0]
+                     for i in range(wl.batch)])
+    return a.alpha_star.cpu().numpy().astype(np.float64), b.alpha_star.cpu().numpy().astype(np.float64), want
+
+
+@pytest.mark.parametrize("n,sigma,V", [(2, 0.25, 50257), (8, 1.0, 50257), (32, 2.0, 50257), (4, 1.0, 129), (16, 0.5, 7001)])
+def test_whole_vocabulary_alpha_star_bucket_search_equals_the_sort(n, sigma, V):
+    wl = W.config4(n, 0, sigma, batch=24, device="cuda", V=V, seed=500 + n)
+    a, b, want = _alpha_both_ways(wl)
+    assert np.abs(a - want).max() <= ALPHA_TOL, (a, want)
+    assert np.abs(b - want).max() <= ALPHA_TOL, (b, want)
+    assert np.abs(a - b).max() <= 2e-7          # (both are stored as fp32)
+
+
+def test_whole_vocabulary_alpha_star_rows_the_buckets_cannot_separate():
+    """Rows built so that the candidate buckets overflow: all ratios equal (draft = target: one bucket holds the
+    row), and ratios on a few levels only (thousands of ties per bucket).  Those rows take the sort; the answers
+    still agree with the oracle."""
+    wl = W.config4(4, 0, 1.0, batch=6, device="cuda", V=20000, seed=77)
+    q = wl.q_logits.clone(); p = wl.p_logits.clone()
+    p[0] = q[0]                                              # identical rows: alpha* = 1
+    p[1] = q[1] + 3.0                                        # a constant shift changes nothing
+    lev = torch.randint(0, 3, (wl.V,), device=q.device).float()
+    p[2] = q[2] + lev                                        # three ratio levels
+    p[3] = q[3] + 0.5 * torch.randint(0, 40, (wl.V,), device=q.device).float()
+    import dataclasses
+    wl2 = dataclasses.replace(wl, q_logits=q, p_logits=p)
+    a, b, want = _alpha_both_ways(wl2)
+    assert abs(want[0] - 1.0) < 1e-12 and abs(want[1] - 1.0) < 1e-12
+    assert np.abs(a - want).max() <= ALPHA_TOL, (a, want)
+    assert np.abs(b - want).max() <= ALPHA_TOL, (b, want)
+
+
 def test_n32_with_a_dominant_draft_token_converges():
     """n = 32: tokens holding a large share of the draft mass need the multiplied-out leave-one-out products
     (the series division loses too many digits there); every instance must converge, and match the oracle."""
