@@ -25,7 +25,8 @@
 #include "gr_verify.cuh"
 
 // The translation unit that includes this file chooses the padded support size: 64 (96-thread CTAs, four per
-// SM) or 128 (128-thread CTAs, one per SM), and a namespace of its own for the instantiation.
+// SM) or 128 (256-thread CTAs, one per SM: its shared memory admits no second CTA, so the one CTA brings two warps
+// per scheduler itself), and a namespace of its own for the instantiation.
 #ifndef GR_FAST_MP
 #define GR_FAST_MP 64
 #define GR_FAST_NS fast64
@@ -36,7 +37,7 @@ namespace GR_FAST_NS {
 
 constexpr int kMP = GR_FAST_MP;       // padded support size of these kernels
 constexpr int kRL = kMP / 32;         // rows (or tokens) per lane when a warp covers the whole support
-constexpr int kFT = kMP == 64 ? 96 : 128;   // threads per CTA (at least kMP - 8: one thread per panel row)
+constexpr int kFT = kMP == 64 ? 96 : 256;   // threads per CTA (at least kMP - 8: one thread per panel row)
 constexpr int kFCtas = kMP == 64 ? 4 : 1;   // CTAs per SM the kernels are compiled for
 constexpr int kFW = kFT / 32;         // warps per CTA
 constexpr int kJC = kMP == 64 ? 6 : 4;      // Hessian nodes staged per chunk
@@ -65,7 +66,7 @@ struct FastLayout {
         g2 = o; o += KP; col = o; o += kMP;
         gw = o; o += kFW * KP; g2w = o; o += kFW * KP;
         tq = o; o += kFMaxNodes; cq = o; o += kFMaxNodes;
-        scal = o; o += 32;
+        scal = o; o += 48;
         uni = o;
         // union: staging of the Hessian operands (two float arrays [kJC * NT][kMS]) / vectors of the Newton step
         const int stage_doubles = (2 * kJC * NT * kMS * 4 + 7) / 8;
@@ -86,7 +87,8 @@ struct FSm {
     GR_PTR(int) id, blk, itmp, trunc;
     int KP;
 };
-enum { SC_Q = 0, SC_FAIL = 1, SC_RED = 8 };
+enum { SC_Q = 0, SC_FAIL = 1, SC_RED = 8, SC_GRID = 24 };   // (SC_RED: one slot per warp; 16..23: preparation outputs;
+                                                            //  SC_GRID: two slots per warp)
 
 __device__ __forceinline__ double ipow(double x, int n) {
     double r = 1.0;
@@ -417,7 +419,7 @@ __device__ void fast_eval(const FSm& sm, int m, int n, GR_PTR(const double) d, d
 static __device__ void fast_grid(const FSm& sm, int m, int n, int slack, double qstep)
 {
     const int tid = threadIdx.x;
-    GR_PTR(double) red = sm.scal + SC_RED;
+    GR_PTR(double) red = sm.scal + SC_GRID;
     double a = 0.0;
     if (tid < m) { a = sm.alpha[tid]; sm.w[tid] = exp(a); }
     // extreme alphas in one pass (they give the extreme weights)
@@ -865,7 +867,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
     sm.col = GR_MKPTR(double, base + L.col, kMP, ck);
     sm.gw = GR_MKPTR(double, base + L.gw, kFW * KP, ck); sm.g2w = GR_MKPTR(double, base + L.g2w, kFW * KP, ck);
     sm.tq = GR_MKPTR(double, base + L.tq, kFMaxNodes, ck); sm.cq = GR_MKPTR(double, base + L.cq, kFMaxNodes, ck);
-    sm.scal = GR_MKPTR(double, base + L.scal, 32, ck);
+    sm.scal = GR_MKPTR(double, base + L.scal, 48, ck);
     sm.J = GR_MKPTR(double, base + L.uni, L.uni_doubles, ck);
     sm.AS = GR_MKPTR(float, reinterpret_cast<float*>(base + L.uni), kJC * NT * kMS, ck);
     sm.HS = GR_MKPTR(float, reinterpret_cast<float*>(base + L.uni) + kJC * NT * kMS, kJC * NT * kMS, ck);
