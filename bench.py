@@ -62,17 +62,58 @@ def _peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed region runs: a thread that polls NVML every few
+    milliseconds (reading only), so that a timed region of a few tens of milliseconds still gets samples; where the
+    NVML binding is missing, `nvidia-smi -lms` in a child process (which starts too slowly for short runs).
+    Samples taken between mark_begin() and mark_end() are the ones reported; with none in there, all of them."""
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
 
-    def __init__(self, index: int):
+    def __init__(self, index: int, uuid: str = None):
         self.index = index
-        self.rows = []
+        self.uuid = uuid
+        self.samples = []          # (host time, sm MHz, set of reasons)
+        self.smax = None
         self.proc = None
         self.thread = None
+        self.stop_flag = False
+        self.t0 = None
+        self.t1 = None
+        self.kind = None
 
     def start(self):
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            h = None
+            if self.uuid:
+                try:
+                    h = pynvml.nvmlDeviceGetHandleByUUID(self.uuid if self.uuid.startswith("GPU-") else "GPU-" + self.uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(self.index)
+            self.smax = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            bits = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40, "sw_power_cap": 0x4}
+            get_reasons = getattr(pynvml, "nvmlDeviceGetCurrentClocksEventReasons",
+                                  getattr(pynvml, "nvmlDeviceGetCurrentClocksThrottleReasons", None))
+
+            def poll():
+                while not self.stop_flag:
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        mask = int(get_reasons(h)) if get_reasons else 0
+                        self.samples.append((time.perf_counter(), mhz, {n for n, b in bits.items() if mask & b}))
+                    except Exception:
+                        pass
+                    time.sleep(0.003)
+            self.kind = "nvml"
+            self.thread = threading.Thread(target=poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            pass
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
                                           "--format=csv,noheader,nounits", "-lms", "20"],
@@ -80,37 +121,50 @@ class ClockSampler:
         except Exception:
             self.proc = None
             return
+        self.kind = "nvidia-smi"
         self.thread = threading.Thread(target=self._read, daemon=True)
         self.thread.start()
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append(line.strip())
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, smax, reasons = [], None, set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
-            parts = [x.strip() for x in r.split(",")]
+            parts = [x.strip() for x in line.strip().split(",")]
             if len(parts) < 6:
                 continue
             try:
-                sm.append(float(parts[0])); smax = float(parts[1])
+                mhz = float(parts[0]); self.smax = float(parts[1])
             except ValueError:
                 continue
-            for nm, val in zip(names, parts[2:6]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        sm.sort()
-        med = sm[len(sm) // 2] if sm else None
-        return {"sm_mhz": med, "sm_max_mhz": smax, "reasons": sorted(reasons), "samples": len(sm)}
+            self.samples.append((time.perf_counter(), mhz,
+                                 {nm for nm, val in zip(self.NAMES, parts[2:6]) if val.lower().startswith("active")}))
+
+    def mark_begin(self):
+        self.t0 = time.perf_counter()
+
+    def mark_end(self):
+        self.t1 = time.perf_counter()
+
+    def stop(self):
+        if self.kind is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no NVML binding and no nvidia-smi"], "samples": 0}
+        self.stop_flag = True
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        elif self.thread is not None:
+            self.thread.join(timeout=1.0)
+        rows = list(self.samples)
+        inside = [r for r in rows if self.t0 is not None and self.t1 is not None and self.t0 <= r[0] <= self.t1]
+        use = inside if inside else rows
+        sm = sorted(r[1] for r in use)
+        reasons = set()
+        for r in use:
+            reasons |= r[2]
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": self.smax, "reasons": sorted(reasons),
+                "samples": len(sm), "sampled": ("during the timed region" if inside else "around the timed region"),
+                "source": self.kind}
 
 
 def run_reference(args):
@@ -200,7 +254,11 @@ def run_ours(args):
     metric = (METRIC if cfg == 3 else
               f"solve+verify instances/sec at V={wl.V},n={wl.n},top-k={wl.topk if wl.topk else 'V'}")
     # the clock sampler runs from before the warm-up so that short timed regions still have samples
-    sampler = ClockSampler(local)
+    try:
+        uuid = str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        uuid = None
+    sampler = ClockSampler(local, uuid)
     if rank == 0:
         sampler.start()
     ev_scan = torch.cuda.Event(enable_timing=True)
@@ -230,6 +288,7 @@ def run_ours(args):
     scan_ms = []
     start = torch.cuda.Event(enable_timing=True); end = torch.cuda.Event(enable_timing=True)
     barrier()
+    sampler.mark_begin()
     start.record()
     for i in range(K):
         step(evs[i])
@@ -239,6 +298,7 @@ def run_ours(args):
     end.record()
     barrier()
     total_ms = start.elapsed_time(end)
+    sampler.mark_end()
     clocks = sampler.stop() if rank == 0 else None
     solve_ms = [e[0].elapsed_time(e[1]) for e in evs]
     verify_ms = [e[1].elapsed_time(e[2]) for e in evs]
