@@ -71,14 +71,15 @@ extern "C" {
  *              token's law then differs from that target by at most tol in L1.  Smaller
  *              values are honoured down to the quadrature floor of a few 1e-9 at the
  *              default quad_step.)
- *              The faster kernel also stops after a Newton step taken from a point
- *              evaluated on the full quadrature grid when the residual that step leaves
- *              is predicted ten times below tol, in one of two ways: the step's
- *              second-order size s2 = sum_i g_i (delta alpha_i)^2 (the residual after
- *              the step stayed within 3.1 s2 + 3e-9 on every benchmark shape; the
- *              reported gradient norm is then 3 s2), or, after a step that contracted
- *              quadratically (r_k = C r_{k-1}^2, C r_{k-1} < 0.1), C r_k^2 (reported
- *              as such).
+ *              The kernels also stop after a Newton step taken from a point evaluated
+ *              on the full quadrature grid when the residual that step leaves is
+ *              predicted below tol, in one of two ways: the step's second-order size
+ *              s2 = sum_i g_i (delta alpha_i)^2 ten times below tol (the residual after
+ *              such a step stayed within 8.5 s2 + 3e-9 on every shape measured; the
+ *              reported gradient norm is then 3 s2), or, after a step that contracted the
+ *              residual by rho < 0.1, 3 rho r_k below tol (reported: rho r_k).  Neither is
+ *              used when the factorisation of the Newton system left less than 2 % of a
+ *              diagonal entry as its pivot (a system too close to singular in fp32).
  *   max_iters  cap on gradient evaluations per system.            default 40
  *   quad_step  step of the trapezoid rule in the log-time variable used to
  *              evaluate the gradient integral; smaller is more accurate and

@@ -79,7 +79,8 @@ __device__ inline int tri(int i, int l) { return i * (i + 1) / 2 + l; }   // l <
 
 // scal[] slots
 enum { S_WMAX = 0, S_WMIN, S_RNORM, S_RPREV, S_LAM, S_FAIL, S_DMAX, S_MEAN, S_SHI, S_S0, S_STEP, S_H, S_DA, S_DB,
-       S_COARSE };
+       S_COARSE, S_PIVOT };
+constexpr int S_ADD = S_MEAN;      // (slot reused: what was added to every Hessian entry)
 
 // Evaluate g (and, if want_jac, the packed lower triangle of the Hessian) at sm.alpha[0..m).
 // d = draft masses of the system's tokens, hmass = draft mass of everything of higher ratio
@@ -364,6 +365,8 @@ __device__ void cholesky(const Sm& sm, int m)
         __syncthreads();
         const double pj = sm.J[tri(j, j)];
         if (!(pj > 0.0)) { if (tid == 0) sm.scal[S_FAIL] = 1.0; __syncthreads(); return; }
+        // smallest pivot relative to the diagonal entry it came from (S_PIVOT; the caller sets it to 1 beforehand)
+        if (tid == 0) sm.scal[S_PIVOT] = fmin(sm.scal[S_PIVOT], pj / (sm.g[j] - sm.g2[j] + sm.scal[S_ADD]));
         const double inv = 1.0 / sqrt(pj);
         for (int i = j + 1 + tid; i < m; i += kSolveThreads) sm.col[i] = sm.J[tri(i, j)] * inv;
         __syncthreads();
@@ -403,8 +406,10 @@ __device__ void chol_solve(const Sm& sm, int m)
 
 // Newton iteration for one system.  On return sm.w[0..m) holds exp(alpha).
 // Returns the status; *gnorm and *iters receive the final L1 gradient norm and the evaluations spent.
+// `warm`: weights to start from (what the fast kernel reached before it gave the instance up), or a null pointer.
 __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(const double) rhs, double hmass,
-                            int slack, double tol, int max_iters, double qstep, double* gnorm, int* iters)
+                            int slack, double tol, int max_iters, double qstep, double* gnorm, int* iters,
+                            const double* warm = nullptr)
 {
     const int tid = threadIdx.x, n = sm.n, KP = sm.KP;
     GR_PTR(double) red = sm.scal + 16;
@@ -441,6 +446,13 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
         } else {
             a0 = log(rhs[tid] / d[tid]);
         }
+    }
+    if (warm != nullptr) {
+        // usable when every weight is positive and finite and they are not all still at the initial 1
+        const double wv = tid < m ? warm[tid] : 1.0;
+        const int bad = __syncthreads_or(!(wv > 0.0) || !(wv < 1.0e300));
+        const int moved = __syncthreads_or(wv != 1.0);
+        if (!bad && moved && tid < m) a0 = log(wv);
     }
     if (!slack) {
         double mean = block_reduce_sum(tid < m ? a0 : 0.0, red) / (double)m;
@@ -482,6 +494,7 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
             const double add = 1.0 / (double)m;
             for (int e = tid; e < m * (m + 1) / 2; e += kSolveThreads) sm.J[e] += add;
         }
+        if (tid == 0) { sm.scal[S_PIVOT] = 1.0; sm.scal[S_ADD] = slack ? 0.0 : 1.0 / (double)m; }
         __syncthreads();
         cholesky(sm, m);
         const bool fail = sm.scal[S_FAIL] != 0.0;
@@ -529,7 +542,8 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
         // quadrature floor, on every benchmark shape).  Ten times below the tolerance: the step is taken and the
         // iteration stops without another evaluation; the reported norm is then the bound 3 s2.
         const double s2 = block_reduce_sum(tid < m ? sm.g[tid] * sm.delta[tid] * sm.delta[tid] : 0.0, red);
-        if (!fail && !coarse && dm <= 1.0 && 10.0 * s2 < tol) {
+        // (not after a factorisation that cancelled all but a few percent of a diagonal entry: see the fast kernel)
+        if (!fail && !coarse && dm <= 1.0 && 10.0 * s2 < tol && sm.scal[S_PIVOT] > 0.02) {
             if (tid < m) sm.w[tid] = exp(sm.alpha[tid]);
             __syncthreads();
             rn = 3.0 * s2;
@@ -616,6 +630,12 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
         tol = 5.0 * tau;
     }
     GR_PTR(double) dT = sm.key; GR_PTR(double) rT = sm.psi; GR_PTR(int) tmap = sm.itmp;
+    // an instance the fast kernel gave up carries the weights that kernel reached: they are kept (sm.key is free
+    // outside the truncated variant) as the starting point of each system
+    const bool warm = only_flagged && !trunc;
+    if (warm && tid < k) sm.key[tid] = pv.w[tid];
+    __syncthreads();
+    const double* warm_w = warm ? &sm.key[0] : nullptr;
     if (tid < k) pv.w[tid] = trunc ? 0.0 : 1.0;
     // with the drafted tuple at hand only the system it selects is solved
     const int sel = fused ? selected_system(fa.draft + (size_t)b * n, n, k, jstar, sm.id, sm.blk, &s_sel) : -2;
@@ -624,7 +644,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
     if (jstar > 0 && sel < 0) {
         double gn = 0.0; int it = 0;
         if (!trunc) {
-            int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it);
+            int st = solve_system(sm, jstar, sm.d, sm.tg, 0.0, 1, tol, max_iters, qstep, &gn, &it, warm_w);
             if (st != GR_OK) status = GR_NOT_CONVERGED;
             if (tid < jstar) pv.w[tid] = sm.w[tid];
         } else {
@@ -650,7 +670,8 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
                 if (m >= 2 && !wanted) skipped = true;
                 if (m >= 2 && wanted) {
                     double gn; int it;
-                    int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it);
+                    int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it,
+                                          warm_w ? warm_w + lo : nullptr);
                     if (st != GR_OK) status = GR_NOT_CONVERGED;
                     gnorm_total += gn; iters_total += it;
                     if (tid < m) pv.w[lo + tid] = sm.w[tid];

@@ -148,6 +148,24 @@ def test_low_target_temperature_with_a_saturated_token():
     _check(P.compare(wl.rows(list(range(416, 440)))))      # includes the heaviest instance (428)
 
 
+def test_very_low_target_temperature_hands_instances_to_the_fp64_kernel():
+    """Target temperature 0.3 on the headline shape: acceptance ~0.9997, weights up to 1e7.  The fp32 Newton system
+    of the fast kernel runs out of accuracy on some instances; those are finished by the fp64 kernel from the point
+    the fast kernel reached.  Every instance must end converged, with the oracle's structure and a gradient norm
+    within the tolerance at the GPU's weights."""
+    base = W.config3(batch=192, device="cuda", seed=77)
+    g = torch.Generator(device="cuda"); g.manual_seed(78)
+    p = base.q_logits + 0.75 * torch.randn(base.q_logits.shape, generator=g, device="cuda")
+    wl = W._finish("config3 at target temperature 0.3", base.V, base.n, base.topk, 0.3, 1.0, base.q_logits, p, g)
+    rep = P.certify(wl)
+    print(rep.summary())
+    assert rep.n_status_ok == rep.n_inst, rep.summary()
+    assert rep.n_struct_mismatch == 0, (rep.summary(), rep.details[:5])
+    assert rep.alpha_err <= ALPHA_TOL, rep.summary()
+    assert rep.cert_solver_max <= CERT_TOL, (rep.summary(), rep.details[:5])
+    assert rep.n_underreported == 0, (rep.summary(), rep.details[:5])
+
+
 def test_ragged_rows_and_unaligned_vocabulary():
     """V not a multiple of the vector width or of the chunk: scalar head / tail paths."""
     for V, n, k in [(1031, 3, 6), (4099, 2, 4), (50257, 4, 5)]:
