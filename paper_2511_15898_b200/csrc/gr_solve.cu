@@ -436,6 +436,7 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
     }
     // starting point: the single-token balance  w/(1+w) * Pr[i in set(omega)] = rhs
     double a0 = 0.0;
+    bool warm_used = false;
     const double D = block_reduce_sum(tid < m ? d[tid] : 0.0, red);   // draft mass of the system
     if (tid < m) {
         if (slack) {
@@ -453,13 +454,15 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
         const int bad = __syncthreads_or(!(wv > 0.0) || !(wv < 1.0e300));
         const int moved = __syncthreads_or(wv != 1.0);
         if (!bad && moved && tid < m) a0 = log(wv);
+        warm_used = !bad && moved;
     }
     if (!slack) {
         double mean = block_reduce_sum(tid < m ? a0 : 0.0, red) / (double)m;
         a0 -= mean;
     }
     if (tid < m) sm.alpha[tid] = fmin(fmax(a0, -kAlphaClamp), kAlphaClamp);
-    if (tid == 0) { sm.scal[S_RPREV] = 1.0e300; sm.scal[S_LAM] = 1.0; sm.scal[S_COARSE] = 1.0; }
+    // (a point handed over by the fast kernel is close to the solution: the full grid from the first evaluation)
+    if (tid == 0) { sm.scal[S_RPREV] = warm_used ? 5.0e-3 : 1.0e300; sm.scal[S_LAM] = 1.0; sm.scal[S_COARSE] = warm_used ? 0.0 : 1.0; }
     __syncthreads();
 
     int status = GR_NOT_CONVERGED;
