@@ -471,6 +471,9 @@ def run_ours(args):
                    "cache": (f"one input set of {bytes_per_instance * B / 1e9:.2f} GB per batch, re-read every step: "
                              + ("larger than the 126 MB L2, no flush needed" if bytes_per_instance * B > 3e8 else
                                 "SMALLER than L2 (the configuration is that small); the step is not HBM-bound")),
+                   "solver": "library defaults: stop at an L1 gradient norm of 3e-7 per convex program (evaluated, or "
+                             "predicted from the last Newton step), quadrature step 0.4; quality.gnorm_max is the "
+                             "largest norm reported in the batch",
                    "parallelism": f"batch x{world}"},
         "roofline": {"bound": "hbm", "kernel": "whole step (streaming + solve + verify kernels)",
                      "what": "bytes of both logit rows / whole solve+verify step time (the streaming kernel is the "
