@@ -74,13 +74,19 @@ bucket_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int
                     char* __restrict__ params, int pstride, int force_sort, float* __restrict__ alpha_out)
 {
     extern __shared__ __align__(16) unsigned char bk_smem[];
-    unsigned long long* bt = reinterpret_cast<unsigned long long*>(bk_smem);     // target mass, then exclusive prefix
-    unsigned long long* bd = bt + kBkBuckets;                                     // draft mass, then exclusive prefix
-    int* cnt = reinterpret_cast<int*>(bd + kBkBuckets);                           // elements per bucket / fill cursor
-    int* seg = cnt + kBkBuckets;                                                  // start of a candidate's segment, -1
-    double* ckey = reinterpret_cast<double*>(seg + kBkBuckets);                   // candidate elements: key,
-    int* cid = reinterpret_cast<int*>(ckey + kBkMaxCand);                         // id,
-    int* sid = cid + kBkMaxCand;                                                  // ids in order
+    GR_CHECK_FLAG_DECL;
+    GR_CHECK_FLAG_INIT;
+    unsigned long long* const bt_raw = reinterpret_cast<unsigned long long*>(bk_smem);
+    int* const cnt_raw = reinterpret_cast<int*>(bt_raw + 2 * kBkBuckets);
+    double* const ckey_raw = reinterpret_cast<double*>(cnt_raw + 2 * kBkBuckets);
+    int* const cid_raw = reinterpret_cast<int*>(ckey_raw + kBkMaxCand);
+    GR_PTR(unsigned long long) bt = GR_MKPTR(unsigned long long, bt_raw, kBkBuckets, GR_CHECK_FLAG);   // target mass, then exclusive prefix
+    GR_PTR(unsigned long long) bd = GR_MKPTR(unsigned long long, bt_raw + kBkBuckets, kBkBuckets, GR_CHECK_FLAG);   // draft mass, ditto
+    GR_PTR(int) cnt = GR_MKPTR(int, cnt_raw, kBkBuckets, GR_CHECK_FLAG);            // elements per bucket / fill cursor
+    GR_PTR(int) seg = GR_MKPTR(int, cnt_raw + kBkBuckets, kBkBuckets, GR_CHECK_FLAG);   // start of a candidate's segment, -1
+    GR_PTR(double) ckey = GR_MKPTR(double, ckey_raw, kBkMaxCand, GR_CHECK_FLAG);    // candidate elements: key,
+    GR_PTR(int) cid = GR_MKPTR(int, cid_raw, kBkMaxCand, GR_CHECK_FLAG);            // id,
+    GR_PTR(int) sid = GR_MKPTR(int, cid_raw + kBkMaxCand, kBkMaxCand, GR_CHECK_FLAG);   // ids in order
     __shared__ double s_r[4][kBkThreads / 32];
     __shared__ unsigned long long s_w[kBkThreads / 32];
     __shared__ int s_nelem, s_fallback;
@@ -235,11 +241,16 @@ bucket_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int
         __syncthreads();
         for (int w2 = 0; w2 < kBkThreads / 32; w2++) best = fmin(best, s_r[0][w2]);
     }
+    __syncthreads();
     if (tid == 0) {
         flag[0] = 0;
         hdr->alpha_star = 1.0 + best;
         hdr->resid_total = -best;
         alpha_out[b] = (float)(1.0 + best);
+        if (GR_CHECK_VALUE) {                       // (bounds-checked build: an access was out of range)
+            hdr->status = GR_CHECK_FAILED;
+            alpha_out[b] = nanf("");
+        }
     }
 }
 

@@ -41,6 +41,9 @@ cases = [("config1", W.config1(batch=16, device="cuda"), None),
          ("headline shape, robust kernel", W.config3(batch=3, device="cuda", seed=3102), G.Options(force_robust=1)),
          ("headline shape, tau=0.05", W.config3(batch=4, device="cuda", seed=3103), G.Options(tau=0.05)),
          ("whole vocabulary V=5000", W.config4(4, 0, 1.0, batch=3, device="cuda", V=5000, seed=99), None),
+         ("whole vocabulary V=50257 (bucket search)", W.config4(8, 0, 1.0, batch=2, device="cuda", seed=98), None),
+         ("whole vocabulary V=5000 (sort)", W.config4(4, 0, 1.0, batch=2, device="cuda", V=5000, seed=97),
+          G.Options(force_robust=1)),
          ("bf16 V=9001", W.config5(batch=4, device="cuda", V=9001, rows_per_pass=4), None)]
 for name, wl, opt in cases:
     s = G.solve(wl.q_logits, wl.p_logits, wl.n, wl.topk, wl.temp_target, wl.temp_draft, opt)
