@@ -616,38 +616,44 @@ static __device__ void fast_newton_step(const FSm& sm, int m, GR_PTR(const doubl
         if (lane < m) yf[lane] = y0;
         if (lane + 32 < m) yf[lane + 32] = y1;
     }
-    if (tid < 32 && kRL != 2) {
-        const int lane = tid;
-        float y[kRL], rd[kRL], an[kRL];
+    if (kRL != 2) {
+        // Wider supports: blocked, eight unknowns at a time from the last panel down.  Every thread keeps its own entry
+        // of the right-hand side in a register; the block's eight entries go through shared memory (two buffers in
+        // turn, one barrier per block), every thread solves the 8 x 8 triangle redundantly and takes the block's
+        // unknowns out of its own entry.  About 350 cycles per block, where the one-warp form above spent over 400
+        // per unknown at four entries per lane.
+        float yl = tid < m ? yf[tid] : 0.f;
+        int buf = 0;
+        for (int j0 = ((m - 1) >> 3) << 3; j0 >= 0; j0 -= 8) {
+            const int nb = min(8, m - j0);
+            GR_PTR(float) yb = yv + 8 * buf;
+            if (tid >= j0 && tid < j0 + nb) yb[tid - j0] = yl;
+            __syncthreads();
+            float x[8];
 #pragma unroll
-        for (int u = 0; u < kRL; u++) {
-            const int l = lane + 32 * u;
-            y[u] = l < m ? yf[l] : 0.f;
-            rd[u] = l < m ? 1.f / dg[l] : 0.f;
-            an[u] = Jm[(m - 1) * kJS + l];
-        }
-        for (int e = m - 1; e >= 0; e--) {
-            float a[kRL];
+            for (int c = 7; c >= 0; c--) {
+                float v = 0.f;
+                if (c < nb) {
+                    v = yb[c];
 #pragma unroll
-            for (int u = 0; u < kRL; u++) a[u] = an[u];
-            if (e > 0) {
-#pragma unroll
-                for (int u = 0; u < kRL; u++) an[u] = Jm[(e - 1) * kJS + lane + 32 * u];
+                    for (int c2 = 7; c2 > c; c2--)
+                        if (c2 < nb) v = fmaf(-Jm[(j0 + c2) * kJS + j0 + c], x[c2], v);
+                    v = v / dg[j0 + c];
+                }
+                x[c] = v;
             }
-            float xv = 0.f;
+            if (tid < j0) {
 #pragma unroll
-            for (int u = 0; u < kRL; u++) xv = (e >> 5) == u ? y[u] * rd[u] : xv;
-            const float xe = __shfl_sync(0xffffffffu, xv, e & 31);
-#pragma unroll
-            for (int u = 0; u < kRL; u++) {
-                const int l = lane + 32 * u;
-                if (l == e) y[u] = xe;
-                else if (l < e) y[u] = fmaf(-a[u], xe, y[u]);
+                for (int c = 0; c < 8; c++)
+                    if (c < nb) yl = fmaf(-Jm[(j0 + c) * kJS + tid], x[c], yl);
             }
-        }
+            if (tid == kFT - 1) {
 #pragma unroll
-        for (int u = 0; u < kRL; u++)
-            if (lane + 32 * u < m) yf[lane + 32 * u] = y[u];
+                for (int c = 0; c < 8; c++)
+                    if (c < nb) yf[j0 + c] = x[c];
+            }
+            buf ^= 1;
+        }
     }
     __syncthreads();
     if (tid < m) sm.delta[tid] = (double)yf[tid];
