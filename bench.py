@@ -500,6 +500,7 @@ def run_ours(args):
                     "status_ok": int((status == 0).sum()), "status_not_converged": int((status == 1).sum()),
                     "status_no_rule": int((status == 2).sum()),
                     "iterations_histogram": np.bincount(iters, minlength=1).tolist()[:64],
+                    "gnorm_predicted": int(rule.gnorm_predicted.sum().item()),
                     "gnorm_max": float(rule.gnorm.max()), "parity_vs_oracle": parity, "wall_ms_total": total_ms},
     }
     print(json.dumps(out), flush=True)

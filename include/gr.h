@@ -257,6 +257,8 @@ int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, 
  *   resid  [batch,kcap] double outer residual r_i (0 on H*)
  *   flow   [batch,kcap] double p_i = tgt_i - r_i
  *   header [batch,8] double: k, jstar, nblocks, alpha_star, gnorm, iterations, lse of the target row, status
+ *          (iterations = gradient evaluations spent, plus 65536 when the gradient norm of at least one of the
+ *          instance's convex programs is a prediction from its last Newton step rather than an evaluation)
  */
 int gr_read_rule(const void* params, int batch, int kcap, int* ids, int* block, double* w,
                  double* resid, double* flow, double* header, void* stream);

@@ -308,9 +308,10 @@ class Rule:
     nblocks: torch.Tensor
     alpha_star: torch.Tensor   # [B] float64
     gnorm: torch.Tensor
-    iters: torch.Tensor
+    iters: torch.Tensor        # gradient evaluations spent
     lse_target: torch.Tensor
     status: torch.Tensor
+    gnorm_predicted: torch.Tensor = None   # [B] bool: the norm of some system was predicted from its last Newton step
 
 
 def read_rule(solved: Solved) -> Rule:
@@ -329,7 +330,7 @@ def read_rule(solved: Solved) -> Rule:
     _check(rc, "gr_read_rule")
     hd = hd.cpu()
     return Rule(ids.cpu(), blk.cpu(), w.cpu(), r.cpu(), p.cpu(), hd[:, 0].long(), hd[:, 1].long(), hd[:, 2].long(),
-                hd[:, 3], hd[:, 4], hd[:, 5].long(), hd[:, 6], hd[:, 7].long())
+                hd[:, 3], hd[:, 4], hd[:, 5].long() & 0xffff, hd[:, 6], hd[:, 7].long(), (hd[:, 5].long() >> 16) & 1 == 1)
 
 
 @dataclasses.dataclass

@@ -72,11 +72,18 @@ struct __align__(16) Header {
     const void* q_row;        // this instance's target row
     int dtype, head;          // logits element type; elements before the first 16-byte boundary
     float temp_target;
-    int iters;                // gradient evaluations spent
+    int iters;                // gradient evaluations spent (low 16 bits); bit 16: the norm of some system is a prediction
     int kcap;                 // capacity of the per-support arrays
     int stride;               // bytes from one instance's header to the next
 };
 static_assert(sizeof(Header) == 96, "params header layout");
+// The evaluation count a system's solver returns carries, in bit 16, whether its last gradient norm was predicted
+// from the final Newton step instead of evaluated; per instance the counts add up and the bits are or-ed.
+constexpr int kItersMask = 0xffff;
+constexpr int kItersPredicted = 1 << 16;
+__host__ __device__ inline int add_iters(int total, int it) {
+    return (((total & kItersMask) + (it & kItersMask)) & kItersMask) | ((total | it) & ~kItersMask);
+}
 
 // Per-instance params block: Header, then
 //   int    id[kcap]     token id in ratio order (position 0 = largest drf/tgt)

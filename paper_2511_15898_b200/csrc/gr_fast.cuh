@@ -775,7 +775,8 @@ __device__ int fast_system(const FSm& sm, int m, int n, GR_PTR(const double) d, 
     double rn = 0.0, rprev = 1.0e300, lam = 1.0;
     bool was_coarse = true;
     bool full_grid_only = false;         // set once a factorisation has failed
-    int stalls = 0;                      // times a step could not be made to reduce the residual at any length tried
+    int stalls = 0;
+    bool predicted = false;              // the norm returned is a prediction, not an evaluation                      // times a step could not be made to reduce the residual at any length tried
     for (; it < max_iters; it++) {
         // far from the solution the trapezoid step is doubled (quadrature error ~4e-6, far below the gradient
         // norm there): half the nodes, every one of them a Hessian node.  Convergence is only ever declared on
@@ -857,6 +858,7 @@ __device__ int fast_system(const FSm& sm, int m, int n, GR_PTR(const double) d, 
             __syncthreads();
             rn = by_step ? kFPredictBound * s2 : rho * rn;
             status = GR_OK; it++;
+            predicted = true;
             break;
         }
     }
@@ -867,7 +869,7 @@ __device__ int fast_system(const FSm& sm, int m, int n, GR_PTR(const double) d, 
         __syncthreads();
     }
     *gnorm = rn;
-    *iters = it;
+    *iters = it | (predicted ? kItersPredicted : 0);
     return status;
 }
 
@@ -956,7 +958,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
                 if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
             }
         }
-        gnorm_total += gn; iters_total += it;
+        gnorm_total += gn; iters_total = add_iters(iters_total, it);
         __syncthreads();
     }
     int lo = jstar;
@@ -973,7 +975,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
                 const int st = fast_system<NT, TPL>(sm, m, n, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep,
                                                     &gn, &it);
                 if (st != GR_OK) status = kNeedFallback;
-                gnorm_total += gn; iters_total += it;
+                gnorm_total += gn; iters_total = add_iters(iters_total, it);
                 if (tid < m) pv.w[lo + tid] = sm.w[tid];
                 __syncthreads();
             }
@@ -989,7 +991,7 @@ fast_solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int ps
                 double gn; int it;
                 const int st = fast_system<NT, TPL>(sm, mT, n, dT, rT, hT, 0, tol, max_iters, qstep, &gn, &it);
                 if (st != GR_OK) status = kNeedFallback;
-                gnorm_total += gn; iters_total += it;
+                gnorm_total += gn; iters_total = add_iters(iters_total, it);
                 if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
             }
             __syncthreads();

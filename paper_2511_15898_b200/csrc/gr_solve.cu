@@ -551,6 +551,7 @@ __device__ int solve_system(const Sm& sm, int m, GR_PTR(const double) d, GR_PTR(
             __syncthreads();
             rn = 3.0 * s2;
             status = GR_OK; it++;
+            it |= kItersPredicted;
             break;
         }
     }
@@ -658,7 +659,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
                 if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
             }
         }
-        gnorm_total += gn; iters_total += it;
+        gnorm_total += gn; iters_total = add_iters(iters_total, it);
         __syncthreads();
     }
     {
@@ -676,7 +677,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
                     int st = solve_system(sm, m, sm.d + lo, sm.p + lo, sm.Dr[lo], 0, tol, max_iters, qstep, &gn, &it,
                                           warm_w ? warm_w + lo : nullptr);
                     if (st != GR_OK) status = GR_NOT_CONVERGED;
-                    gnorm_total += gn; iters_total += it;
+                    gnorm_total += gn; iters_total = add_iters(iters_total, it);
                     if (tid < m) pv.w[lo + tid] = sm.w[tid];
                     __syncthreads();
                 }
@@ -692,7 +693,7 @@ solve_kernel(const char* __restrict__ ws, char* __restrict__ params, int pstride
                     double gn; int it;
                     int st = solve_system(sm, mT, dT, rT, hT, 0, tol, max_iters, qstep, &gn, &it);
                     if (st != GR_OK) status = GR_NOT_CONVERGED;
-                    gnorm_total += gn; iters_total += it;
+                    gnorm_total += gn; iters_total = add_iters(iters_total, it);
                     if (tid < mT) pv.w[tmap[tid]] = sm.w[tid];
                 }
                 __syncthreads();

@@ -53,6 +53,7 @@ def _check_cert(rep: P.CertReport, max_near_tie_frac=0.02, CERT_TOL=CERT_TOL):
     assert rep.lse_err_max <= LSE_TOL, rep.summary()
     assert rep.cert_max <= CERT_TOL + LSE_TOL, (rep.summary(), rep.details[:5])
     assert rep.n_underreported == 0, (rep.summary(), rep.details[:5])
+    assert rep.n_evaluated_off == 0, (rep.summary(), rep.details[:5])
     assert rep.n_status_ok == rep.n_inst, rep.summary()
     assert rep.n_near_tie <= max(1, int(max_near_tie_frac * rep.n_inst)), rep.summary()
 
