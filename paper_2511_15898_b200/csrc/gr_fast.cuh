@@ -554,10 +554,16 @@ static __device__ void fast_newton_step(const FSm& sm, int m, GR_PTR(const doubl
         const int t0 = j0 + 8;
         if (t0 < m) {
             const int lane = tid & 31, warp = tid >> 5, gid = lane >> 2, tig = lane & 3;
-            int t = 0;
-            for (int mi = 0; t0 + 16 * mi < m; mi++) {
-                for (int ni = 0; ni <= 2 * mi + 1 && t0 + 8 * ni < m; ni++, t++) {
-                    if (t % kFW != warp) continue;
+            // tile t of the lower triangle: row mi of 16-row tiles holds tiles mi (mi + 1) .. (mi + 1)(mi + 2) - 1
+            // (2 mi + 2 of them); each warp takes every kFW-th tile and finds (mi, ni) from t directly
+            const int nmt = (m - t0 + 15) >> 4;
+            for (int t = warp; t < nmt * (nmt + 1); t += kFW) {
+                int mi = (int)((sqrtf((float)(4 * t + 1)) - 1.f) * 0.5f);
+                while (mi * (mi + 1) > t) mi--;
+                while ((mi + 1) * (mi + 2) <= t) mi++;
+                const int ni = t - mi * (mi + 1);
+                {
+                    if (t0 + 8 * ni >= m) continue;
                     const int ra = t0 + 16 * mi + gid, rb = ra + 8, l0 = t0 + 8 * ni, cb = l0 + gid;
                     const bool oa = ra < m, ob = rb < m, oc = cb < m;
                     const float fa[4] = {oa ? -Jm[ra * kJS + j0 + tig] : 0.f, ob ? -Jm[rb * kJS + j0 + tig] : 0.f,
