@@ -77,7 +77,8 @@ extern "C" {
  *              s2 = sum_i g_i (delta alpha_i)^2 ten times below tol (the residual after
  *              such a step stayed within 8.5 s2 + 3e-9 on every shape measured; the
  *              reported gradient norm is then 3 s2), or, after a step that contracted the
- *              residual by rho < 0.1, 3 rho r_k below tol (reported: rho r_k).  Neither is
+ *              residual by rho < 0.1, 3 rho r_k below tol (reported: rho r_k; the faster
+ *              kernels only).  Neither is
  *              used when the factorisation of the Newton system left less than 2 % of a
  *              diagonal entry as its pivot (a system too close to singular in fp32).
  *   max_iters  cap on gradient evaluations per system.            default 40
