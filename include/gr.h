@@ -239,8 +239,9 @@ int gr_solve_verify(const void* q_logits, const void* p_logits, int dtype, int V
  *   workspace   scratch of gr_workspace_bytes(V, 1, topk, batch) bytes, 16-byte aligned.
  *   alpha_star  out [batch, n_count] float, row-major; NaN where status is not GR_OK.
  *   status      out [batch]: GR_OK or GR_BAD_LOGITS.
- * Supports as for the rule: top-k up to GR_MAX_SUPPORT, or the whole vocabulary when V <= GR_MAX_SUPPORT;
- * an untruncated draft on a larger vocabulary returns GR_E_TOO_LARGE (gr_solve still gives its alpha*).
+ * Supports: top-k up to GR_MAX_SUPPORT, or the whole vocabulary of any size (beyond GR_MAX_SUPPORT tokens
+ * the minimum of psi is searched per draft count without sorting the row, as in gr_solve); a top-k beyond
+ * GR_MAX_SUPPORT on a larger vocabulary returns GR_E_TOO_LARGE.
  * Other return values as gr_solve.
  */
 #define GR_MAX_ALPHA_N 8

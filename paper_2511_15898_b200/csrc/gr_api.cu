@@ -104,7 +104,8 @@ static int solve_impl(const void* q_logits, const void* p_logits, int dtype, int
         // psi, or with force_robust a sort of the whole row and a prefix scan)
         char* scratch = (char*)workspace + (size_t)gr::ws_stride() * (size_t)batch;
         gr::launch_fullsort(q_logits, p_logits, dtype, V, n, (double)temp_target, (double)temp_draft, batch,
-                            (const char*)workspace, scratch, (char*)params, pstride, force_robust, alpha_star, st);
+                            (const char*)workspace, scratch, (char*)params, pstride, force_robust, alpha_star, 1, 0,
+                            nullptr, st);
     }
     if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
     return GR_OK;
@@ -147,9 +148,21 @@ int gr_alpha_star(const void* q_logits, const void* p_logits, int dtype, int V, 
     if (((uintptr_t)q_logits & 15) || ((uintptr_t)p_logits & 15) || ((uintptr_t)workspace & 15)) return GR_E_ALIGN;
     const int kfull = (topk <= 0 || topk >= V) ? V : topk;
     const int kcap = gr::kcap_of(V, topk);
-    if (kcap == 0) return GR_E_TOO_LARGE;
+    if (kcap == 0 && kfull != V) return GR_E_TOO_LARGE;       // a truncated support beyond the capacity
     cudaStream_t st = (cudaStream_t)stream;
     gr::NvtxRange whole("gr_alpha_star");
+    if (kcap == 0) {
+        // untruncated draft on a large vocabulary: the streaming pass for the row statistics, then the bucketed
+        // search for min psi once per draft count (rows it cannot separate take the sort)
+        gr::launch_scan(q_logits, p_logits, dtype, V, kfull, true, (double)temp_target, (double)temp_draft, batch,
+                        (char*)workspace, nullptr, 0, kcap, st);
+        char* scratch = (char*)workspace + (size_t)gr::ws_stride() * (size_t)batch;
+        for (int j = 0; j < n_count; j++)
+            gr::launch_fullsort(q_logits, p_logits, dtype, V, n_list[j], (double)temp_target, (double)temp_draft, batch,
+                                (const char*)workspace, scratch, nullptr, 0, 0, alpha_star, n_count, j, status, st);
+        if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return GR_E_LAUNCH; }
+        return GR_OK;
+    }
     gr::launch_scan(q_logits, p_logits, dtype, V, kfull, false, (double)temp_target, (double)temp_draft, batch,
                     (char*)workspace, nullptr, 0, kcap, st);
     gr::launch_alpha((const char*)workspace, V, topk, (double)temp_target, (double)temp_draft, n_list, n_count, batch,

@@ -71,7 +71,8 @@ template <typename T>
 __global__ void __launch_bounds__(kBkThreads)
 bucket_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int n, double temp_t, double temp_d,
                     const char* __restrict__ ws, char* __restrict__ scratch, size_t scratch_stride,
-                    char* __restrict__ params, int pstride, int force_sort, float* __restrict__ alpha_out)
+                    char* __restrict__ params, int pstride, int force_sort, float* __restrict__ alpha_out,
+                    int out_stride, int out_off, int* __restrict__ status_out)
 {
     extern __shared__ __align__(16) unsigned char bk_smem[];
     GR_CHECK_FLAG_DECL;
@@ -93,10 +94,15 @@ bucket_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long b = blockIdx.x;
     const WsHeader* wh = reinterpret_cast<const WsHeader*>(ws + (size_t)b * ws_stride());
-    Header* hdr = reinterpret_cast<Header*>(params + (size_t)b * pstride);
+    // (no params block and a status array when called for the optimal acceptance alone)
+    Header* hdr = params ? reinterpret_cast<Header*>(params + (size_t)b * pstride) : nullptr;
     int* flag = reinterpret_cast<int*>(scratch + (size_t)b * scratch_stride);
+    if (tid == 0 && status_out) status_out[b] = wh->bad != 0 ? GR_BAD_LOGITS : GR_OK;
     if (wh->bad != 0 || force_sort) {
-        if (tid == 0) flag[0] = 1;                  // (a bad row returns at once there too)
+        if (tid == 0) {
+            flag[0] = 1;                            // (a bad row returns at once there too)
+            if (wh->bad != 0 && status_out) alpha_out[(size_t)b * out_stride + out_off] = nanf("");
+        }
         return;
     }
     const T* qrow = q + (size_t)b * V;
@@ -244,12 +250,12 @@ bucket_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int
     __syncthreads();
     if (tid == 0) {
         flag[0] = 0;
-        hdr->alpha_star = 1.0 + best;
-        hdr->resid_total = -best;
-        alpha_out[b] = (float)(1.0 + best);
+        if (hdr) { hdr->alpha_star = 1.0 + best; hdr->resid_total = -best; }
+        alpha_out[(size_t)b * out_stride + out_off] = (float)(1.0 + best);
         if (GR_CHECK_VALUE) {                       // (bounds-checked build: an access was out of range)
-            hdr->status = GR_CHECK_FAILED;
-            alpha_out[b] = nanf("");
+            if (hdr) hdr->status = GR_CHECK_FAILED;
+            if (status_out) status_out[b] = GR_CHECK_FAILED;
+            alpha_out[(size_t)b * out_stride + out_off] = nanf("");
         }
     }
 }
@@ -258,7 +264,7 @@ template <typename T>
 __global__ void __launch_bounds__(kFsThreads)
 fullsort_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, int n, double temp_t, double temp_d,
                       const char* __restrict__ ws, char* __restrict__ scratch, char* __restrict__ params, int pstride,
-                      float* __restrict__ alpha_out)
+                      float* __restrict__ alpha_out, int out_stride, int out_off)
 {
     __shared__ double s_a[kFsThreads / 32], s_b[kFsThreads / 32];
     __shared__ double s_carry[2];
@@ -266,8 +272,8 @@ fullsort_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, i
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long b = blockIdx.x;
     const WsHeader* wh = reinterpret_cast<const WsHeader*>(ws + (size_t)b * ws_stride());
-    Header* hdr = reinterpret_cast<Header*>(params + (size_t)b * pstride);
-    if (wh->bad != 0) return;                       // header already says GR_BAD_LOGITS
+    Header* hdr = params ? reinterpret_cast<Header*>(params + (size_t)b * pstride) : nullptr;
+    if (wh->bad != 0) return;                       // header / status already say GR_BAD_LOGITS
     const T* qrow = q + (size_t)b * V;
     const T* prow = p + (size_t)b * V;
     const int VP = next_pow2(V);
@@ -411,15 +417,14 @@ fullsort_alpha_kernel(const T* __restrict__ q, const T* __restrict__ p, int V, i
     __syncthreads();
     if (tid == 0) {
         for (int w2 = 1; w2 < kFsThreads / 32; w2++) best = fmin(best, s_min[w2]);
-        hdr->alpha_star = 1.0 + best;
-        hdr->resid_total = -best;
-        alpha_out[b] = (float)(1.0 + best);
+        if (hdr) { hdr->alpha_star = 1.0 + best; hdr->resid_total = -best; }
+        alpha_out[(size_t)b * out_stride + out_off] = (float)(1.0 + best);
     }
 }
 
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
                      const char* ws, char* scratch, char* params, int pstride, int force_sort, float* alpha_out,
-                     cudaStream_t st)
+                     int out_stride, int out_off, int* status_out, cudaStream_t st)
 {
     // function attributes belong to the device: set once per device (a failure shows up as a launch error)
     static bool configured[kMaxDevices] = {false};
@@ -440,20 +445,23 @@ void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, doub
     if (dtype == GR_F32)
         bucket_alpha_kernel<float><<<batch, kBkThreads, kBkSmemBytes, st>>>((const float*)q, (const float*)p, V, n, temp_t,
                                                                             temp_d, ws, scratch, sstride, params, pstride,
-                                                                            force_sort, alpha_out);
+                                                                            force_sort, alpha_out, out_stride, out_off,
+                                                                            status_out);
     else
         bucket_alpha_kernel<__nv_bfloat16><<<batch, kBkThreads, kBkSmemBytes, st>>>((const __nv_bfloat16*)q,
                                                                                     (const __nv_bfloat16*)p, V, n, temp_t,
                                                                                     temp_d, ws, scratch, sstride, params,
-                                                                                    pstride, force_sort, alpha_out);
+                                                                                    pstride, force_sort, alpha_out, out_stride,
+                                                                                    out_off, status_out);
     if (dtype == GR_F32)
         fullsort_alpha_kernel<float><<<batch, kFsThreads, kFsSmemBytes, st>>>((const float*)q, (const float*)p, V, n, temp_t,
-                                                                   temp_d, ws, scratch, params, pstride, alpha_out);
+                                                                   temp_d, ws, scratch, params, pstride, alpha_out,
+                                                                   out_stride, out_off);
     else
         fullsort_alpha_kernel<__nv_bfloat16><<<batch, kFsThreads, kFsSmemBytes, st>>>((const __nv_bfloat16*)q,
                                                                            (const __nv_bfloat16*)p, V, n, temp_t,
                                                                            temp_d, ws, scratch, params, pstride,
-                                                                           alpha_out);
+                                                                           alpha_out, out_stride, out_off);
 }
 
 }  // namespace gr

@@ -29,7 +29,7 @@ int launch_solve_any(const char* ws, char* params, int pstride, int kcap, int V,
 size_t fullsort_scratch_bytes(int V);
 void launch_fullsort(const void* q, const void* p, int dtype, int V, int n, double temp_t, double temp_d, int batch,
                      const char* ws, char* scratch, char* params, int pstride, int force_sort, float* alpha_out,
-                     cudaStream_t st);
+                     int out_stride, int out_off, int* status_out, cudaStream_t st);
 void launch_alpha(const char* ws, int V, int topk, double temp_t, double temp_d, const int* n_list, int n_count,
                   int batch, float* alpha_out, int* status_out, cudaStream_t st);
 void launch_verify(const char* params, const int* draft, const float* uni, int batch, int* out_token,

@@ -92,7 +92,7 @@ def test_argument_errors_are_reported_before_any_launch(lib):
                                A, 0)
     assert alpha([]) == -1 and alpha([0]) == -1 and alpha([33]) == -1 and alpha(list(range(1, 10))) == -1
     assert alpha([2], q=0) == -2 and alpha([2], q=A + 4) == -3 and alpha([2], tt=0.0) == -1
-    assert alpha([2], V=100000, topk=0) == -5   # untruncated draft beyond GR_MAX_SUPPORT
+    assert alpha([2], V=100000, topk=500) == -5   # truncated support beyond GR_MAX_SUPPORT
     assert alpha([2, 4], batch=0) == 0
 
 
