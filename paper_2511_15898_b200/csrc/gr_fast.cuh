@@ -789,10 +789,10 @@ __device__ int fast_system(const FSm& sm, int m, int n, GR_PTR(const double) d, 
         // the full grid.
         const bool coarse = rprev > 1.0e-2 && !full_grid_only;
         fast_grid(sm, m, n, slack, coarse ? 2.0 * qstep : qstep);
-        // Hessian nodes: every second one on the full grid; every one on the doubled step, except in the wide kernel,
-        // where a chunk of kJC nodes would leave half of the eight warps without a node (the Hessian only steers, and
-        // its quadrature error at four times the step, ~2e-3 relative, is far below the residual there)
-        fast_eval<NT, TPL>(sm, m, n, d, hmass, true, (coarse && kFW <= kJC) ? 1 : 2);
+        // Hessian nodes: every second one on the full grid, every one on the doubled step (taking every second one
+        // there too kept all eight warps of the wide kernel busy and saved 8 % on one shape, but a Hessian from six or
+        // seven nodes cost others one to three more evaluations, and a 128-token, n = 16 shape seven times its time)
+        fast_eval<NT, TPL>(sm, m, n, d, hmass, true, coarse ? 1 : 2);
         rn = block_reduce_sum(tid < m ? fabs(sm.g[tid] - rhs[tid]) : 0.0, red);
         if (rn <= tol && !coarse) { status = GR_OK; it++; break; }
         // (a residual on the full grid is not compared with the coarse grid's: they differ by the coarse quadrature error)
