@@ -133,6 +133,13 @@ def test_supports_of_65_to_128_tokens(n, topk):
     _check(P.compare(wl))
 
 
+@pytest.mark.parametrize("n,topk", [(32, 128), (24, 64), (17, 100)])
+def test_general_kernel_on_wide_supports_with_more_than_16_drafts(n, topk):
+    """n above 16 takes the general kernel whatever the support: up to sixteen tokens per group in its product tree."""
+    wl = W.config3(batch=3, device="cuda", seed=4000 + n + topk, V=20000, n=n, topk=topk)
+    _check(P.compare(wl))
+
+
 def test_low_target_temperature_with_a_saturated_token():
     """Sharper target (temperature 0.5): acceptance ~0.94 and single tokens that must win nearly every tuple they
     are in (weights up to ~1e5).  Parity on a slice, and on a larger batch every instance converges in few steps."""
